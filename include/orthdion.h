@@ -1,0 +1,129 @@
+/* orthdion.h - C interface of the B200 (sm_100a) Orth-Dion / Dion optimizer-step library.
+ *
+ * One call of orthdion_step performs, for one weight matrix, the step of Algorithm 1 of the
+ * paper ("Orth-Dion / Stripped Dion (one step)"; appendix algorithms "Stripped Dion" and
+ * "Orth-Dion"), written with the letters of this interface:
+ *
+ *     B  = M + G                                 buffer            (Alg. 1 line 1)
+ *     P  = orth(B * Q_prev)                      left factor       (Alg. 1 line 2)
+ *     R  = B^T * P                               right factor      (Alg. 1 line 3)
+ *     Q  = orth(R)   [ORTH]   |  ColNorm(R) [COLNORM]              (Alg. 1 line 4)
+ *     X <- (1 - eta*wd) * X - eta*scale * P * Q^T                  (Alg. 1 lines 5-6)
+ *     M <- a * B - b * P * R^T                   error feedback    (Alg. 1 line 7)
+ *     Q_prev <- Q                                warm start        (Alg. 1 line 8)
+ *
+ * Paper letters: G_t = G, R_t = M (residual), M_t = B, V_{t-1} = Q_prev, U_t = P, W_t = R.
+ * orth(.) is the thin QR factor with a positive diagonal in the triangular factor
+ * (CholeskyQR2 on the device, with a shifted third pass when the Gram matrix is
+ * ill-conditioned).  (a, b) default to (1, 1 - mu); the paper's line 7 is (beta, beta).
+ *
+ * Conventions
+ *  - Every matrix pointer is a DEVICE pointer owned by the caller; matrices are row-major and
+ *    contiguous: X, M, G are m x n (leading dimension n), Q is n x r (leading dimension r).
+ *  - X, M and Q are updated in place; G is only read.  Q holds Q_prev on entry, Q on return.
+ *  - M and Q are float32.  X and G are float32 or bfloat16 (orthdion_set_dtypes).
+ *  - All device pointers must be 16-byte aligned.
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *    synchronising.  The library allocates no device memory: the caller passes a workspace of
+ *    at least orthdion_workspace_bytes*() bytes, 256-byte aligned, which must stay untouched
+ *    until the enqueued work has finished.  P, R and the status words live in it.
+ *  - Return value: 0 on success, a negative ORTHDION_ERR_* code when the host rejects the
+ *    arguments (nothing is enqueued then).  Numerical conditions never trap: they are reported
+ *    per matrix through status flags in the workspace (orthdion_last_status).  A matrix whose
+ *    factorisation fails even after the shifted pass keeps X, M and Q unchanged.
+ *  - Handles are immutable plans apart from the setters and may be shared by any number of
+ *    matrices of the same shape.  Setters must not race with a step call on the same handle.
+ *  - The library needs a CUDA device of compute capability 10.x; there is no CPU fallback.
+ */
+#ifndef ORTHDION_H_
+#define ORTHDION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct orthdion_plan* orthdion_t;
+
+/* Algorithm 1 line 4: which normalisation of the right factor. */
+#define ORTHDION_MODE_ORTH     0   /* Q = orth(R): Orth-Dion                     */
+#define ORTHDION_MODE_COLNORM  1   /* Q = ColNorm(R): (Stripped) Dion            */
+
+#define ORTHDION_DTYPE_F32   0
+#define ORTHDION_DTYPE_BF16  1
+
+/* Which kernels carry the matrix products.  TENSOR: tcgen05 tensor-core kernels with
+ * bf16-split operands and fp32 accumulation in tensor memory.  SIMT: plain fp32 FMA kernels
+ * (any r >= 1; meant for tiny matrices and as an on-device cross-check). */
+#define ORTHDION_ENGINE_TENSOR 0
+#define ORTHDION_ENGINE_SIMT   1
+
+/* host-side error codes */
+#define ORTHDION_OK                 0
+#define ORTHDION_ERR_INVALID_ARG   -1   /* bad handle, count, mode, dtype, engine, scalar       */
+#define ORTHDION_ERR_RANK          -2   /* r < 1, r > min(m, n), or r not supported by engine   */
+#define ORTHDION_ERR_NULL          -3   /* a required pointer is null                           */
+#define ORTHDION_ERR_WORKSPACE     -4   /* workspace too small or misaligned                    */
+#define ORTHDION_ERR_CUDA          -5   /* a CUDA runtime call failed (launch, attribute, ...)  */
+#define ORTHDION_ERR_ALIGNMENT     -6   /* a matrix pointer is not 16-byte aligned              */
+
+/* per-matrix device status flags (bit mask) */
+#define ORTHDION_STATUS_SHIFTED_LEFT    1   /* left QR took the shifted three-pass path         */
+#define ORTHDION_STATUS_SHIFTED_RIGHT   2   /* right QR took the shifted three-pass path        */
+#define ORTHDION_STATUS_RANK_DEFICIENT  4   /* factorisation failed: X, M, Q left unchanged     */
+#define ORTHDION_STATUS_NONFINITE       8   /* a Gram matrix held Inf/NaN: treated as failure   */
+#define ORTHDION_STATUS_ZERO_COLUMN    16   /* COLNORM met a zero column of R (kept zero)       */
+#define ORTHDION_STATUS_WAIT_LIMIT     32   /* a bounded device-side wait expired (kernel bug)  */
+
+/* Create a plan for m x n matrices at rank r (Algorithm 1 "REQUIRE" line: step size eta, EF
+ * coefficient; mu gives the default (a, b) = (1, 1 - mu)).  Defaults: X and G bfloat16,
+ * scale = 1, engine TENSOR.  The TENSOR engine needs r % 16 == 0, n % 8 == 0; SIMT any r.
+ * Host memory only. */
+int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r,
+                    float mu, float eta, float wd, int32_t mode);
+int orthdion_destroy(orthdion_t h);
+
+int orthdion_set_dtypes(orthdion_t h, int32_t x_dtype, int32_t g_dtype);
+int orthdion_set_lr(orthdion_t h, float eta);               /* eta_t of a schedule               */
+int orthdion_set_scale(orthdion_t h, float scale);          /* extra factor on the update; 1.0   */
+int orthdion_set_ef(orthdion_t h, float a, float b);        /* M <- a*B - b*P*R^T                */
+int orthdion_set_engine(orthdion_t h, int32_t engine);
+/* Number of bf16 split terms products are built from (1 = plain bf16, 3 = three products of a
+ * two-term split, about 2^-16 relative accuracy).  which: 0 = B*Q and B^T*P, 1 = Gram/apply of
+ * the QR, 2 = P*R^T of the error feedback, 3 = P*Q^T of the weight update. <=0 restores default. */
+int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes);
+
+/* Workspace sizes in bytes (host computation, no CUDA call). */
+size_t orthdion_workspace_bytes(orthdion_t h);
+size_t orthdion_workspace_bytes_grouped(const orthdion_t* hs, int32_t count);
+
+/* One step for one matrix (Algorithm 1). */
+int orthdion_step(orthdion_t h, void* X, float* M, const void* G, float* Q,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* One step for `count` matrices; hs[i] is the plan of matrix i.  X, M, G, Q are HOST arrays of
+ * `count` device pointers.  Matrices are packed by equal plan parameters ("sort-and-pack"
+ * batching, appendix on the wide-model study) and every stage runs once per pack.  Results per
+ * matrix are identical to orthdion_step. */
+int orthdion_step_grouped(const orthdion_t* hs, int32_t count,
+                          void* const* X, float* const* M, const void* const* G, float* const* Q,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* Device pointers to the factors P (m x r) and R (n x r) that the last step left in the
+ * workspace (for checks).  index = position in the grouped call, 0 for orthdion_step. */
+int orthdion_get_factors(const orthdion_t* hs, int32_t count, int32_t index, void* workspace,
+                         const float** P, const float** R);
+
+/* Copies the `count` status words of the last step to host `flags` (synchronises `stream`). */
+int orthdion_last_status(const orthdion_t* hs, int32_t count, void* workspace, void* stream,
+                         int32_t* flags);
+
+/* Library/kernels self-description: returns a static string naming the build (arch, engines). */
+const char* orthdion_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ORTHDION_H_ */

@@ -1,0 +1,389 @@
+// Host side of liborthdion: plans, workspace layout, sort-and-pack batching and the stage
+// sequence of one optimizer step.  All device work is enqueued on the caller's stream.
+#include "../../include/orthdion.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "common.cuh"
+#include "factor_kernels.cuh"
+#include "simt_kernels.cuh"
+#include "tensor_engine.cuh"
+
+using namespace od;
+
+struct orthdion_plan {
+    uint32_t magic;
+    int64_t m, n;
+    int32_t r;
+    float mu, eta, wd, scale, ef_a, ef_b;
+    int32_t mode, x_dtype, g_dtype, engine;
+    int32_t passes[4];
+};
+
+namespace {
+
+constexpr uint32_t kMagic = 0x0D10A5E7u;
+constexpr int32_t kMaxRank = 1024;
+constexpr size_t kScratchBudget = (size_t)24 << 30;   // per launch batch
+constexpr float kShiftRel = 1e-5f;
+constexpr float kCondLimit = 1024.f;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool valid(orthdion_t h) { return h && h->magic == kMagic; }
+
+bool same_class(const orthdion_plan* a, const orthdion_plan* b) {
+    return a->m == b->m && a->n == b->n && a->r == b->r && a->mode == b->mode &&
+           a->x_dtype == b->x_dtype && a->g_dtype == b->g_dtype && a->engine == b->engine &&
+           a->eta == b->eta && a->wd == b->wd && a->scale == b->scale && a->ef_a == b->ef_a &&
+           a->ef_b == b->ef_b && std::memcmp(a->passes, b->passes, sizeof(a->passes)) == 0;
+}
+
+// Per-matrix scratch carving (byte offsets).  kmax = max(m, n).
+struct Scratch {
+    int64_t gram, linv, tmpA, tmpB;
+    TensorScratch ts;
+    size_t bytes;
+};
+
+Scratch scratch_layout(const orthdion_plan* p) {
+    Scratch s{};
+    const size_t rr = align_up((size_t)p->r * p->r * 4, 256);
+    const size_t kr = align_up((size_t)std::max(p->m, p->n) * p->r * 4, 256);
+    size_t off = 0;
+    s.gram = off; off += rr;
+    s.linv = off; off += rr;
+    s.tmpA = off; off += kr;
+    s.tmpB = off; off += kr;
+    if (p->engine == ORTHDION_ENGINE_TENSOR) off = tensor_scratch_layout(p->m, p->n, p->r, off, &s.ts);
+    s.bytes = align_up(off, 256);
+    return s;
+}
+
+struct Batching {
+    std::vector<std::vector<int>> batches;   // matrix indices per launch batch, class by class
+    size_t scratch_bytes = 0;                // max over batches
+};
+
+Batching make_batches(const orthdion_t* hs, int32_t count) {
+    Batching out;
+    std::vector<char> done(count, 0);
+    for (int i = 0; i < count; ++i) {
+        if (done[i]) continue;
+        std::vector<int> cls;
+        for (int j = i; j < count; ++j)
+            if (!done[j] && same_class(hs[i], hs[j])) { cls.push_back(j); done[j] = 1; }
+        const size_t per = scratch_layout(hs[i]).bytes;
+        size_t cap = std::max<size_t>(1, kScratchBudget / std::max<size_t>(per, 1));
+        cap = std::min<size_t>(cap, MAXB);
+        const size_t nb = (cls.size() + cap - 1) / cap;
+        const size_t bs = (cls.size() + nb - 1) / nb;
+        for (size_t b = 0; b < cls.size(); b += bs) {
+            std::vector<int> one(cls.begin() + b, cls.begin() + std::min(cls.size(), b + bs));
+            out.scratch_bytes = std::max(out.scratch_bytes, one.size() * per);
+            out.batches.push_back(std::move(one));
+        }
+    }
+    return out;
+}
+
+// Workspace: [status words][P_0 R_0][P_1 R_1]...[scratch of the largest batch]
+struct Layout {
+    std::vector<size_t> p_off, r_off;
+    size_t status_off = 0, scratch_off = 0, total = 0;
+};
+
+Layout make_layout(const orthdion_t* hs, int32_t count, size_t scratch_bytes) {
+    Layout l;
+    size_t off = align_up((size_t)count * 4, 256);
+    l.p_off.resize(count);
+    l.r_off.resize(count);
+    for (int i = 0; i < count; ++i) {
+        l.p_off[i] = off; off += align_up((size_t)hs[i]->m * hs[i]->r * 4, 256);
+        l.r_off[i] = off; off += align_up((size_t)hs[i]->n * hs[i]->r * 4, 256);
+    }
+    l.scratch_off = off;
+    l.total = off + scratch_bytes;
+    return l;
+}
+
+#define CU_CHECK(expr)                                                     \
+    do {                                                                   \
+        cudaError_t e__ = (expr);                                          \
+        if (e__ != cudaSuccess) {                                          \
+            std::fprintf(stderr, "orthdion: %s failed: %s\n", #expr, cudaGetErrorString(e__)); \
+            return ORTHDION_ERR_CUDA;                                      \
+        }                                                                  \
+    } while (0)
+
+int ensure_attributes() {
+    static int state = 0;   // 0 unknown, 1 ok, -1 failed
+    if (state) return state > 0 ? 0 : ORTHDION_ERR_CUDA;
+    cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)CH_SMEM_BYTES);
+    if (e == cudaSuccess) e = tensor_engine_set_attributes();
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "orthdion: kernel attribute setup failed: %s\n", cudaGetErrorString(e));
+        state = -1;
+        return ORTHDION_ERR_CUDA;
+    }
+    state = 1;
+    return 0;
+}
+
+template <class RA, class RB, class EP>
+void launch_simt(const Batch& b, int64_t Md, int64_t Nd, int64_t Kd, RA ra, RB rb, EP ep, cudaStream_t st) {
+    dim3 grid((unsigned)((Nd + 63) / 64), (unsigned)((Md + 63) / 64), (unsigned)b.count);
+    simt_gemm_kernel<RA, RB, EP><<<grid, 256, 0, st>>>(b, Md, Nd, Kd, ra, rb, ep);
+}
+
+Sel sel(int where, int64_t off = 0) { return Sel{where, 0, off}; }
+
+// ---- tall-skinny QR of `in` (rows x r) into `fin` (CholeskyQR2; third pass when flagged) -------
+void qr_stage(const orthdion_plan* p, const Batch& b, const Scratch& sc, Sel in, int64_t rows, Sel fin,
+              int which, cudaStream_t st) {
+    const int r = p->r;
+    const int shift_bit = which ? ST_SHIFT_R : ST_SHIFT_L;
+    const Sel gram = sel(W_SCRATCH, sc.gram), linv = sel(W_SCRATCH, sc.linv);
+    const Sel tmpA = sel(W_SCRATCH, sc.tmpA), tmpB = sel(W_SCRATCH, sc.tmpB);
+    const bool tensor = p->engine == ORTHDION_ENGINE_TENSOR;
+    for (int pass = 1; pass <= 3; ++pass) {
+        const Sel src = pass == 1 ? in : (pass == 2 ? tmpA : tmpB);
+        const int only_shift = pass == 3;
+        // Gram = src^T src
+        if (tensor) {
+            tensor_gram(p->m, p->n, r, p->passes[1], b, sc.ts, src, rows, gram, only_shift ? shift_bit : 0, st);
+        } else {
+            EpStore eg{gram, gram, only_shift ? shift_bit : 0, 1, r, only_shift};
+            launch_simt(b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, st);
+        }
+        CholArgs ca{gram, linv, r, which, pass, kShiftRel, kCondLimit};
+        chol_inv_kernel<<<b.count, CH_THREADS, CH_SMEM_BYTES, st>>>(b, ca);
+        // dst = src * L^{-T}
+        EpStore ea{};
+        if (pass == 1) ea = EpStore{tmpA, tmpA, 0, 1, r, 0};
+        else if (pass == 2) ea = EpStore{fin, tmpB, shift_bit, 1, r, 0};
+        else ea = EpStore{fin, fin, shift_bit, 1, r, 1};
+        if (tensor) {
+            tensor_apply(p->m, p->n, r, p->passes[1], b, sc.ts, src, rows, linv, ea, st);
+        } else {
+            launch_simt(b, rows, r, r, RdPlain{src, r, 1}, RdPlain{linv, r, 1}, ea, st);
+        }
+    }
+}
+
+void run_batch(const orthdion_plan* p, const Batch& b, const Scratch& sc, cudaStream_t st) {
+    const int64_t m = p->m, n = p->n;
+    const int r = p->r;
+    const int gb = p->g_dtype == ORTHDION_DTYPE_BF16, xb = p->x_dtype == ORTHDION_DTYPE_BF16;
+    const bool tensor = p->engine == ORTHDION_ENGINE_TENSOR;
+    const float c = 1.f - p->eta * p->wd, d = p->eta * p->scale;
+    const Sel sP = sel(W_P), sR = sel(W_R), sQ = sel(W_Q);
+
+    // Alg. 1 lines 1-2:  Y = (M + G) Q_prev   -> P slot
+    if (tensor) tensor_k1(m, n, r, gb, p->passes[0], b, sc.ts, st);
+    else launch_simt(b, m, r, n, RdBuffer{n, gb, 0}, RdPlain{sQ, 1, r}, EpStore{sP, sP, 0, 0, r, 0}, st);
+    qr_stage(p, b, sc, sP, m, sP, 0, st);
+    // Alg. 1 line 3:  R = (M + G)^T P
+    if (tensor) tensor_k3(m, n, r, gb, p->passes[0], b, sc.ts, st);
+    else launch_simt(b, n, r, m, RdBuffer{n, gb, 1}, RdPlain{sP, 1, r}, EpStore{sR, sR, 0, 0, r, 0}, st);
+    // Alg. 1 line 4
+    if (p->mode == ORTHDION_MODE_ORTH) {
+        qr_stage(p, b, sc, sR, n, sQ, 1, st);
+    } else {
+        dim3 grid((unsigned)((r + 31) / 32), 1, (unsigned)b.count);
+        colnorm_kernel<<<grid, 1024, 0, st>>>(b, n, r);
+    }
+    // Alg. 1 lines 5-7:  M <- a B - b P R^T ;  X <- c X - d P Q^T
+    if (tensor) {
+        tensor_k5(m, n, r, gb, xb, p->passes[2], p->passes[3], p->ef_a, p->ef_b, c, d, b, sc.ts, st);
+    } else {
+        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sR, r, 1}, EpErrorFeedback{p->ef_a, p->ef_b, n, gb}, st);
+        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sQ, r, 1}, EpWeights{c, d, n, xb}, st);
+    }
+}
+
+int check_ptr(const void* p) {
+    if (!p) return ORTHDION_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(p) % 16) return ORTHDION_ERR_ALIGNMENT;
+    return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r, float mu, float eta, float wd,
+                    int32_t mode) {
+    if (!out) return ORTHDION_ERR_NULL;
+    *out = nullptr;
+    if (m < 1 || n < 1 || m > (1 << 24) || n > (1 << 24)) return ORTHDION_ERR_INVALID_ARG;
+    if (mode != ORTHDION_MODE_ORTH && mode != ORTHDION_MODE_COLNORM) return ORTHDION_ERR_INVALID_ARG;
+    if (!(mu == mu) || !(eta == eta) || !(wd == wd)) return ORTHDION_ERR_INVALID_ARG;
+    if (r < 1 || r > m || r > n || r > kMaxRank) return ORTHDION_ERR_RANK;
+    orthdion_plan* p = new orthdion_plan();
+    p->magic = kMagic;
+    p->m = m; p->n = n; p->r = r;
+    p->mu = mu; p->eta = eta; p->wd = wd; p->scale = 1.f;
+    p->ef_a = 1.f; p->ef_b = 1.f - mu;
+    p->mode = mode;
+    p->x_dtype = ORTHDION_DTYPE_BF16; p->g_dtype = ORTHDION_DTYPE_BF16;
+    p->engine = tensor_engine_supports(m, n, r) ? ORTHDION_ENGINE_TENSOR : ORTHDION_ENGINE_SIMT;
+    p->passes[0] = 3; p->passes[1] = 3; p->passes[2] = 3; p->passes[3] = 1;
+    *out = p;
+    return ORTHDION_OK;
+}
+
+int orthdion_destroy(orthdion_t h) {
+    if (!valid(h)) return ORTHDION_ERR_INVALID_ARG;
+    h->magic = 0;
+    delete h;
+    return ORTHDION_OK;
+}
+
+int orthdion_set_dtypes(orthdion_t h, int32_t x_dtype, int32_t g_dtype) {
+    if (!valid(h)) return ORTHDION_ERR_INVALID_ARG;
+    if ((x_dtype != ORTHDION_DTYPE_F32 && x_dtype != ORTHDION_DTYPE_BF16) ||
+        (g_dtype != ORTHDION_DTYPE_F32 && g_dtype != ORTHDION_DTYPE_BF16))
+        return ORTHDION_ERR_INVALID_ARG;
+    h->x_dtype = x_dtype; h->g_dtype = g_dtype;
+    // an fp32 weight matrix shows the update at full precision: build P Q^T from split terms too
+    h->passes[3] = (x_dtype == ORTHDION_DTYPE_F32) ? 3 : 1;
+    return ORTHDION_OK;
+}
+
+int orthdion_set_lr(orthdion_t h, float eta) {
+    if (!valid(h) || !(eta == eta)) return ORTHDION_ERR_INVALID_ARG;
+    h->eta = eta;
+    return ORTHDION_OK;
+}
+
+int orthdion_set_scale(orthdion_t h, float scale) {
+    if (!valid(h) || !(scale == scale)) return ORTHDION_ERR_INVALID_ARG;
+    h->scale = scale;
+    return ORTHDION_OK;
+}
+
+int orthdion_set_ef(orthdion_t h, float a, float b) {
+    if (!valid(h) || !(a == a) || !(b == b)) return ORTHDION_ERR_INVALID_ARG;
+    h->ef_a = a; h->ef_b = b;
+    return ORTHDION_OK;
+}
+
+int orthdion_set_engine(orthdion_t h, int32_t engine) {
+    if (!valid(h)) return ORTHDION_ERR_INVALID_ARG;
+    if (engine == ORTHDION_ENGINE_SIMT) { h->engine = engine; return ORTHDION_OK; }
+    if (engine != ORTHDION_ENGINE_TENSOR) return ORTHDION_ERR_INVALID_ARG;
+    if (!tensor_engine_supports(h->m, h->n, h->r)) return ORTHDION_ERR_RANK;
+    h->engine = engine;
+    return ORTHDION_OK;
+}
+
+int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes) {
+    if (!valid(h) || which < 0 || which > 3) return ORTHDION_ERR_INVALID_ARG;
+    if (passes <= 0) {
+        passes = (which == 3) ? (h->x_dtype == ORTHDION_DTYPE_F32 ? 3 : 1) : 3;
+    } else if (passes != 1 && passes != 3) {
+        return ORTHDION_ERR_INVALID_ARG;
+    }
+    h->passes[which] = passes;
+    return ORTHDION_OK;
+}
+
+size_t orthdion_workspace_bytes_grouped(const orthdion_t* hs, int32_t count) {
+    if (!hs || count < 1) return 0;
+    for (int i = 0; i < count; ++i)
+        if (!valid(hs[i])) return 0;
+    Batching bt = make_batches(hs, count);
+    return make_layout(hs, count, bt.scratch_bytes).total;
+}
+
+size_t orthdion_workspace_bytes(orthdion_t h) { return orthdion_workspace_bytes_grouped(&h, 1); }
+
+int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, float* const* M,
+                          const void* const* G, float* const* Q, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+    if (!hs || !X || !M || !G || !Q || !workspace) return ORTHDION_ERR_NULL;
+    if (count < 1) return ORTHDION_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i) {
+        if (!valid(hs[i])) return ORTHDION_ERR_INVALID_ARG;
+        int e;
+        if ((e = check_ptr(X[i])) || (e = check_ptr(M[i])) || (e = check_ptr(G[i])) || (e = check_ptr(Q[i])))
+            return e;
+    }
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return ORTHDION_ERR_WORKSPACE;
+    Batching bt = make_batches(hs, count);
+    Layout lay = make_layout(hs, count, bt.scratch_bytes);
+    if (workspace_bytes < lay.total) return ORTHDION_ERR_WORKSPACE;
+    int e = ensure_attributes();
+    if (e) return e;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = reinterpret_cast<char*>(workspace);
+    Batch* b = new Batch();
+    int rc = ORTHDION_OK;
+    for (const auto& idx : bt.batches) {
+        const orthdion_plan* p = hs[idx[0]];
+        const Scratch sc = scratch_layout(p);
+        b->count = (int32_t)idx.size();
+        b->pad = 0;
+        for (size_t k = 0; k < idx.size(); ++k) {
+            const int i = idx[k];
+            MatWork& w = b->w[k];
+            w.X = X[i]; w.M = M[i]; w.G = G[i]; w.Q = Q[i];
+            w.P = reinterpret_cast<float*>(ws + lay.p_off[i]);
+            w.R = reinterpret_cast<float*>(ws + lay.r_off[i]);
+            w.status = reinterpret_cast<int32_t*>(ws + lay.status_off) + i;
+            w.scratch = ws + lay.scratch_off + k * sc.bytes;
+        }
+        init_status_kernel<<<1, MAXB, 0, st>>>(*b);
+        run_batch(p, *b, sc, st);
+        cudaError_t ce = cudaGetLastError();
+        if (ce != cudaSuccess) {
+            std::fprintf(stderr, "orthdion: launch failed: %s\n", cudaGetErrorString(ce));
+            rc = ORTHDION_ERR_CUDA;
+            break;
+        }
+    }
+    delete b;
+    return rc;
+}
+
+int orthdion_step(orthdion_t h, void* X, float* M, const void* G, float* Q, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+    void* const xs[1] = {X};
+    float* const ms[1] = {M};
+    const void* const gs[1] = {G};
+    float* const qs[1] = {Q};
+    return orthdion_step_grouped(&h, 1, xs, ms, gs, qs, workspace, workspace_bytes, stream);
+}
+
+int orthdion_get_factors(const orthdion_t* hs, int32_t count, int32_t index, void* workspace,
+                         const float** P, const float** R) {
+    if (!hs || !workspace || !P || !R) return ORTHDION_ERR_NULL;
+    if (count < 1 || index < 0 || index >= count) return ORTHDION_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i)
+        if (!valid(hs[i])) return ORTHDION_ERR_INVALID_ARG;
+    Layout lay = make_layout(hs, count, 0);
+    char* ws = reinterpret_cast<char*>(workspace);
+    *P = reinterpret_cast<const float*>(ws + lay.p_off[index]);
+    *R = reinterpret_cast<const float*>(ws + lay.r_off[index]);
+    return ORTHDION_OK;
+}
+
+int orthdion_last_status(const orthdion_t* hs, int32_t count, void* workspace, void* stream, int32_t* flags) {
+    if (!hs || !workspace || !flags) return ORTHDION_ERR_NULL;
+    if (count < 1) return ORTHDION_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    CU_CHECK(cudaMemcpyAsync(flags, workspace, (size_t)count * 4, cudaMemcpyDeviceToHost, st));
+    CU_CHECK(cudaStreamSynchronize(st));
+    return ORTHDION_OK;
+}
+
+const char* orthdion_version(void) {
+    return "orthdion sm_100a: engines tensor(tcgen05, bf16-split) + simt(fp32)";
+}
+
+}  // extern "C"

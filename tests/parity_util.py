@@ -1,0 +1,81 @@
+"""Helpers for the GPU-vs-oracle parity tests: run the CUDA library and the float64 oracle on the
+same seeded tensors and compare what the benchmark spec's tolerance is stated on."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import orthdion_oracle as orc
+from paper_2605_16341_b200 import binding as od
+from paper_2605_16341_b200 import workloads as wl
+
+TOL_STEP = 1e-4       # ||dX_gpu - dX_or||_F / ||dX_or||_F after one step from identical state
+TOL_CHAIN = 1e-3      # the same after 10 chained steps
+TOL_ORTHO = 1e-5      # max |Q^T Q - I|
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().double().cpu().numpy()
+
+
+def rel(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+class GpuMatrix:
+    """One matrix on the GPU with its plan and workspace."""
+
+    def __init__(self, spec, X, M, Q, *, mu, eta, wd=0.0, mode=od.MODE_ORTH, engine=None, ef=None,
+                 scale=None, passes=None):
+        self.spec = spec
+        self.h = od.orthdion_create(spec.m, spec.n, spec.r, mu, eta, wd, mode)
+        od.orthdion_set_dtypes(self.h, spec.x_dtype, spec.g_dtype)
+        if engine is not None:
+            od.orthdion_set_engine(self.h, engine)
+        if ef is not None:
+            od.orthdion_set_ef(self.h, *ef)
+        if scale is not None:
+            od.orthdion_set_scale(self.h, scale)
+        for k, v in (passes or {}).items():
+            od.orthdion_set_passes(self.h, k, v)
+        self.X, self.M, self.Q = X.cuda().contiguous(), M.cuda().contiguous(), Q.cuda().contiguous()
+        self.ws = od.alloc_workspace(od.orthdion_workspace_bytes(self.h))
+        self.eta, self.wd, self.scale = eta, wd, 1.0 if scale is None else scale
+
+    def step(self, G):
+        self.G = G.cuda().contiguous()
+        od.orthdion_step(self.h, self.X, self.M, self.G, self.Q, self.ws)
+        torch.cuda.synchronize()
+
+    def factors(self):
+        return od.orthdion_get_factors([self.h], 0, self.ws, (self.spec.m, self.spec.n, self.spec.r))
+
+    def status(self):
+        return od.orthdion_last_status([self.h], self.ws)[0]
+
+    def close(self):
+        od.orthdion_destroy(self.h)
+
+
+def delta_x_from_factors(P, Q, X_before, eta, wd, scale):
+    """dX formed in float64 from the GPU's fp32 factors (what the weight update applies before
+    the storage rounding of X)."""
+    return -eta * scale * (f64(P) @ f64(Q).T) - eta * wd * f64(X_before)
+
+
+def check_bf16_rounding(X_after, X_before, P, Q, eta, wd, scale, sample=4096, seed=0):
+    """Stored bf16 weights equal the rounded fp32 result up to one bf16 ulp on sampled entries."""
+    g = np.random.default_rng(seed)
+    m, n = X_after.shape
+    ii, jj = g.integers(0, m, sample), g.integers(0, n, sample)
+    Pn, Qn = f64(P), f64(Q)
+    d = np.einsum("ik,ik->i", Pn[ii], Qn[jj])
+    xb = f64(X_before)[ii, jj]
+    exact = (1.0 - eta * wd) * xb - eta * scale * d
+    got = f64(X_after)[ii, jj]
+    ulp = np.maximum(np.abs(exact), 2.0 ** -126) * 2.0 ** -7
+    return float(np.max(np.abs(got - exact) / ulp))
+
+
+def oracle_mode(mode):
+    return orc.ORTH if mode == od.MODE_ORTH else orc.COLNORM

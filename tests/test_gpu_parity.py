@@ -1,0 +1,281 @@
+"""GPU-vs-oracle parity of the optimizer step, through the C-ABI, element by element.
+
+Tolerances (the benchmark spec): one step from identical state  ||dX_gpu - dX_or||_F / ||dX_or||_F <= 1e-4,
+<= 1e-3 after 10 chained steps (GPU carries its own fp32 M, Q; the oracle float64), and
+max |Q^T Q - I| <= 1e-5.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import orthdion_oracle as orc
+from paper_2605_16341_b200 import binding as od
+from paper_2605_16341_b200 import workloads as wl
+
+from parity_util import (TOL_CHAIN, TOL_ORTHO, TOL_STEP, GpuMatrix, check_bf16_rounding,
+                         delta_x_from_factors, f64, oracle_mode, rel)
+
+pytestmark = pytest.mark.gpu
+
+ENGINES = [od.ENGINE_SIMT, od.ENGINE_TENSOR]
+ENGINE_IDS = ["simt", "tensor"]
+MODES = [od.MODE_ORTH, od.MODE_COLNORM]
+F32, BF16 = torch.float32, torch.bfloat16
+
+
+def make_problem(m, n, r, xdt, gdt, seed, m_scale=0.3):
+    spec = wl.MatrixSpec("t", m, n, r, xdt, gdt)
+    g = torch.Generator().manual_seed(seed)
+    X = (0.02 * torch.randn(m, n, generator=g)).to(xdt)
+    M = m_scale * torch.randn(m, n, generator=g)
+    G = torch.randn(m, n, generator=g).to(gdt)
+    Q = wl.random_orthonormal(n, r, g)
+    return spec, X, M, G, Q
+
+
+def one_step_compare(spec, X, M, G, Q, *, mode, engine, mu=0.95, eta=0.01, wd=0.0, ef=None, scale=None,
+                     tol=TOL_STEP):
+    gm = GpuMatrix(spec, X, M, Q, mu=mu, eta=eta, wd=wd, mode=mode, engine=engine, ef=ef, scale=scale)
+    gm.step(G)
+    assert gm.status() & ~(od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT) == 0
+    kw = dict(ef=ef) if ef is not None else dict(mu=mu)
+    ref = orc.step(f64(X), f64(M), f64(G), f64(Q), eta=eta, wd=wd, scale=1.0 if scale is None else scale,
+                   mode=oracle_mode(mode), **kw)
+    P, R = gm.factors()
+    sc = 1.0 if scale is None else scale
+    dx_ref = ref["X"] - f64(X)
+    if spec.x_dtype == F32:
+        dx_gpu = f64(gm.X) - f64(X)
+    else:
+        dx_gpu = delta_x_from_factors(P, gm.Q, X, eta, wd, sc)
+        assert check_bf16_rounding(gm.X, X, P, gm.Q, eta, wd, sc) <= 1.0 + 1e-6
+    errs = dict(dx=rel(dx_gpu, dx_ref), M=rel(f64(gm.M), ref["M"]), Q=rel(f64(gm.Q), ref["Q"]),
+                P=rel(f64(P), ref["P"]), R=rel(f64(R), ref["R"]))
+    assert errs["dx"] <= tol, errs
+    assert errs["M"] <= tol, errs
+    assert errs["P"] <= tol and errs["R"] <= tol and errs["Q"] <= tol, errs
+    Pn = f64(P)
+    assert np.abs(Pn.T @ Pn - np.eye(spec.r)).max() <= TOL_ORTHO
+    Qn = f64(gm.Q)
+    if mode == od.MODE_ORTH:
+        assert np.abs(Qn.T @ Qn - np.eye(spec.r)).max() <= TOL_ORTHO
+    else:
+        assert np.abs(np.linalg.norm(Qn, axis=0) - 1.0).max() <= TOL_ORTHO
+    gm.close()
+    return errs
+
+
+# ------------------------------------------------------------------ cfg0: 10 chained steps
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_cfg0_chained_both_modes(engine):
+    w = wl.workload("cfg0")
+    spec = w.matrices[0]
+    m_traj = {}
+    for mode in MODES:
+        X, M, Q = wl.initial_state(spec, 0, 0)
+        gm = GpuMatrix(spec, X, M, Q, mu=w.mu, eta=w.eta, wd=w.wd, mode=mode, engine=engine)
+        Xo, Mo, Qo = f64(X), f64(M), f64(Q)
+        m_traj[mode] = []
+        for t in range(10):
+            G = wl.gradient(w, spec, 0, 0, t, None)
+            x_before_gpu = f64(gm.X)
+            gm.step(G)
+            assert gm.status() == 0
+            ref = orc.step(Xo, Mo, f64(G), Qo, eta=w.eta, mu=w.mu, wd=w.wd, mode=oracle_mode(mode))
+            dx_gpu = f64(gm.X) - x_before_gpu
+            dx_ref = ref["X"] - Xo
+            tol = TOL_STEP if t == 0 else TOL_CHAIN
+            assert rel(dx_gpu, dx_ref) <= tol, (mode, t, rel(dx_gpu, dx_ref))
+            assert rel(f64(gm.M), ref["M"]) <= tol
+            assert rel(f64(gm.X), ref["X"]) <= 1e-5
+            Qn = f64(gm.Q)
+            if mode == od.MODE_ORTH:
+                assert np.abs(Qn.T @ Qn - np.eye(spec.r)).max() <= TOL_ORTHO
+            Xo, Mo, Qo = ref["X"], ref["M"], ref["Q"]
+            m_traj[mode].append(f64(gm.M))
+        gm.close()
+    # Lemma 4.3 on the device: the residual trajectory does not depend on the mode
+    for a, b in zip(m_traj[od.MODE_ORTH], m_traj[od.MODE_COLNORM]):
+        assert rel(a, b) <= 1e-4
+
+
+# ------------------------------------------------------------------ one step, several shapes
+SHAPES_ANY = [(200, 328, 24), (129, 520, 8), (64, 64, 64), (520, 136, 40), (96, 1000, 1), (300, 77, 5)]
+SHAPES_TENSOR = [(256, 512, 16), (384, 640, 64), (200, 328, 48), (1000, 264, 128), (136, 2056, 32),
+                 (640, 384, 272)]
+
+
+@pytest.mark.parametrize("shape", SHAPES_ANY)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dt", [(F32, F32), (BF16, BF16)])
+def test_one_step_simt_shapes(shape, mode, dt):
+    m, n, r = shape
+    spec, X, M, G, Q = make_problem(m, n, r, dt[0], dt[1], seed=m * 7 + n)
+    one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_SIMT)
+
+
+@pytest.mark.parametrize("shape", SHAPES_TENSOR)
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dt", [(F32, F32), (BF16, BF16), (F32, BF16)])
+def test_one_step_tensor_shapes(shape, mode, dt):
+    m, n, r = shape
+    spec, X, M, G, Q = make_problem(m, n, r, dt[0], dt[1], seed=m * 7 + n)
+    one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_TENSOR)
+
+
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_paper_error_feedback_form_and_decay(engine):
+    spec, X, M, G, Q = make_problem(256, 384, 32, F32, F32, seed=3)
+    beta = 0.7
+    gm = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, mode=od.MODE_ORTH, engine=engine, ef=(beta, beta))
+    gm.step(G)
+    ref = orc.step(f64(X), f64(M), f64(G), f64(Q), eta=0.01, ef=(beta, beta))
+    P, _ = gm.factors()
+    # R_{t+1} = beta (I - U U^T) M_t is orthogonal to the left factor (up to fp32 cancellation)
+    assert np.abs(f64(P).T @ f64(gm.M)).max() <= 2e-3 * np.abs(ref["B"]).max() * np.sqrt(spec.m)
+    assert rel(f64(gm.M), ref["M"]) <= TOL_STEP
+    gm.close()
+    one_step_compare(spec, X, M, G, Q, mode=od.MODE_ORTH, engine=engine, wd=0.1, scale=0.5, eta=0.02)
+
+
+# ------------------------------------------------------------------ degenerate inputs
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_zero_buffer_is_flagged_and_state_untouched(engine):
+    spec, X, M, G, Q = make_problem(256, 256, 16, BF16, BF16, seed=5)
+    M.zero_(); G.zero_()
+    gm = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, engine=engine)
+    gm.step(G)
+    assert gm.status() & od.STATUS_RANK_DEFICIENT
+    assert torch.equal(gm.X.cpu(), X) and torch.equal(gm.Q.cpu(), Q) and torch.equal(gm.M.cpu(), M)
+    ref = orc.step(f64(X), f64(M), f64(G), f64(Q), eta=0.01, mu=0.95)
+    assert ref["status"] == orc.STATUS_RANK_DEFICIENT
+    gm.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_nonfinite_gradient_is_flagged_and_state_untouched(engine):
+    spec, X, M, G, Q = make_problem(256, 256, 16, F32, F32, seed=6)
+    G[3, 5] = float("nan")
+    gm = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, engine=engine)
+    gm.step(G)
+    assert gm.status() & (od.STATUS_NONFINITE | od.STATUS_RANK_DEFICIENT)
+    assert torch.equal(gm.X.cpu(), X) and torch.equal(gm.Q.cpu(), Q) and torch.equal(gm.M.cpu(), M)
+    gm.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_ill_conditioned_projection_takes_shifted_path(engine):
+    # B Q_prev with a condition number near 1e6: CholeskyQR2 alone would break down
+    m, n, r = 512, 384, 32
+    g = torch.Generator().manual_seed(7)
+    spec = wl.MatrixSpec("t", m, n, r, F32, F32)
+    U = wl.random_orthonormal(m, r, g)
+    Q = wl.random_orthonormal(n, r, g)
+    s = torch.logspace(0, -6, r)
+    G = ((U * s[None, :]) @ Q.T).contiguous()
+    X = torch.zeros(m, n)
+    M = torch.zeros(m, n)
+    gm = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, engine=engine)
+    gm.step(G)
+    st = gm.status()
+    assert st & od.STATUS_SHIFTED_LEFT and not (st & od.STATUS_RANK_DEFICIENT)
+    P, _ = gm.factors()
+    Pn = f64(P)
+    assert np.isfinite(Pn).all()
+    assert np.abs(Pn.T @ Pn - np.eye(r)).max() <= 1e-4
+    # the well-conditioned leading directions agree with the oracle
+    ref = orc.step(f64(X), f64(M), f64(G), f64(Q), eta=0.01, mu=0.95)
+    assert np.abs(Pn[:, :8] - ref["P"][:, :8]).max() <= 1e-3
+    gm.close()
+
+
+# ------------------------------------------------------------------ grouped == single, resume
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_grouped_matches_single_and_is_deterministic(engine):
+    shapes = [(256, 384, 32), (384, 256, 32), (256, 384, 32), (128, 128, 16), (384, 256, 32), (256, 384, 32)]
+    specs, st, Gs = [], [], []
+    for i, (m, n, r) in enumerate(shapes):
+        spec, X, M, G, Q = make_problem(m, n, r, BF16, BF16, seed=100 + i)
+        specs.append(spec); st.append((X, M, Q)); Gs.append(G)
+    hs = []
+    for spec in specs:
+        h = od.orthdion_create(spec.m, spec.n, spec.r, 0.95, 0.01, 0.0, od.MODE_ORTH)
+        od.orthdion_set_engine(h, engine)
+        hs.append(h)
+    dev = [tuple(t.cuda() for t in s) for s in st]
+    Gd = [g.cuda() for g in Gs]
+    ws = od.alloc_workspace(od.orthdion_workspace_bytes_grouped(hs))
+    table = od.PointerTable(hs, [d[0] for d in dev], [d[1] for d in dev], Gd, [d[2] for d in dev])
+    for _ in range(2):
+        od.orthdion_step_grouped(table, ws)
+    torch.cuda.synchronize()
+    assert od.orthdion_last_status(hs, ws) == [0] * len(hs)
+    for i, spec in enumerate(specs):
+        gm = GpuMatrix(spec, *st[i], mu=0.95, eta=0.01, engine=engine)
+        for _ in range(2):
+            gm.step(Gs[i])
+        assert torch.equal(gm.X, dev[i][0]) and torch.equal(gm.M, dev[i][1]) and torch.equal(gm.Q, dev[i][2])
+        P, R = od.orthdion_get_factors(hs, i, ws, (spec.m, spec.n, spec.r))
+        P1, R1 = gm.factors()
+        assert torch.equal(P, P1) and torch.equal(R, R1)
+        gm.close()
+    for h in hs:
+        od.orthdion_destroy(h)
+
+
+@pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
+def test_state_is_only_m_and_q(engine):
+    # 4 steps in one go == 2 steps, state copied out and back, 2 more steps (bitwise)
+    spec, X, M, G, Q = make_problem(256, 384, 32, BF16, BF16, seed=11)
+    g = torch.Generator().manual_seed(12)
+    Gs = [torch.randn(256, 384, generator=g).to(BF16) for _ in range(4)]
+    a = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, engine=engine)
+    for t in range(4):
+        a.step(Gs[t])
+    b = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, engine=engine)
+    for t in range(2):
+        b.step(Gs[t])
+    c = GpuMatrix(spec, b.X.cpu(), b.M.cpu(), b.Q.cpu(), mu=0.95, eta=0.01, engine=engine)
+    for t in range(2, 4):
+        c.step(Gs[t])
+    assert torch.equal(a.X, c.X) and torch.equal(a.M, c.M) and torch.equal(a.Q, c.Q)
+    for x in (a, b, c):
+        x.close()
+
+
+# ------------------------------------------------------------------ cfg1: 4096 x 4096, r = 256, bf16
+@pytest.mark.parametrize("mode", MODES)
+def test_cfg1_first_steps(mode):
+    w = wl.workload("cfg1")
+    spec = w.matrices[0]
+    X, M, Q = wl.initial_state(spec, 0, 0)
+    basis = wl.grad_basis(w, spec, 0, 0)
+    gm = GpuMatrix(spec, X, M, Q, mu=w.mu, eta=w.eta, wd=w.wd, mode=mode)
+    Xo, Mo, Qo = f64(X), f64(M), f64(Q)
+    for t in range(3):
+        G = wl.gradient(w, spec, 0, 0, t, basis)
+        xb = gm.X.clone()
+        gm.step(G)
+        assert gm.status() == 0
+        ref = orc.step(Xo, Mo, f64(G), Qo, eta=w.eta, mu=w.mu, wd=w.wd, mode=oracle_mode(mode))
+        P, R = gm.factors()
+        dx_gpu = delta_x_from_factors(P, gm.Q, xb, w.eta, w.wd, 1.0)
+        dx_ref = ref["X"] - Xo
+        tol = TOL_STEP if t == 0 else TOL_CHAIN
+        assert rel(dx_gpu, dx_ref) <= tol, (t, rel(dx_gpu, dx_ref))
+        assert rel(f64(gm.M), ref["M"]) <= tol
+        assert check_bf16_rounding(gm.X, xb, P, gm.Q, w.eta, w.wd, 1.0) <= 1.0 + 1e-6
+        Pn, Qn = f64(P), f64(gm.Q)
+        assert np.abs(Pn.T @ Pn - np.eye(spec.r)).max() <= TOL_ORTHO
+        if mode == od.MODE_ORTH:
+            assert np.abs(Qn.T @ Qn - np.eye(spec.r)).max() <= TOL_ORTHO
+        # the oracle carries the bf16-stored weights forward, like the device does
+        Xo, Mo, Qo = f64(gm.X), ref["M"], ref["Q"]
+    gm.close()
+
+
+def test_tensor_engine_rejects_unsupported_rank():
+    h = od.orthdion_create(128, 128, 5, 0.95, 0.01, 0.0, od.MODE_ORTH)
+    with pytest.raises(od.OrthDionError):
+        od.orthdion_set_engine(h, od.ENGINE_TENSOR)
+    od.orthdion_destroy(h)
