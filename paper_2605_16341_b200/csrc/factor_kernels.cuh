@@ -71,6 +71,11 @@ struct CholArgs {
     int32_t pass;    // 1, 2 or 3
     float shift_rel; // shift = shift_rel * trace(Gram) on the retry of pass 1
     float cond_limit;// take the shifted path when max diag(L) / min diag(L) exceeds this (pass 1)
+    // Optional fp32 column sums of squares, colsq[kb * colsq_ld + i], kb < colsq_kb: when given they
+    // replace the Gram diagonal.  (The tensor core truncates when it adds into its fp32 accumulator,
+    // which biases long sums of squares low; the off-diagonal sums have no such bias.)
+    Sel colsq;
+    int32_t colsq_kb, colsq_ld;
 };
 
 // Factor Gram = L L^T (blocked, right-looking) and overwrite `work` with L^{-1}.
@@ -82,6 +87,7 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     float* gemm_smem = reinterpret_cast<float*>(smem_raw);
     float* diag_smem = gemm_smem + CH_GROUPS * 2 * 16 * 65;
     __shared__ float red[32];
+    __shared__ float s_diag[1024];
     __shared__ int s_fail;
     __shared__ float s_trace, s_dmin, s_dmax;
     __shared__ int s_status;
@@ -106,7 +112,18 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     // trace and finiteness of the Gram diagonal
     {
         float t = 0.f;
-        for (int i = tid; i < r; i += CH_THREADS) t += A[(int64_t)i * r + i];
+        for (int i = tid; i < r; i += CH_THREADS) {
+            float d;
+            if (a.colsq_kb > 0) {
+                const float* cs = pick(w, a.colsq);
+                d = 0.f;
+                for (int kb = 0; kb < a.colsq_kb; ++kb) d += cs[(int64_t)kb * a.colsq_ld + i];
+            } else {
+                d = A[(int64_t)i * r + i];
+            }
+            s_diag[i] = d;
+            t += d;
+        }
         for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
         if (lane == 0) red[warp] = t;
         __syncthreads();
@@ -131,7 +148,7 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         for (int64_t e = tid; e < (int64_t)r * r; e += CH_THREADS) {
             int i = (int)(e / r), j = (int)(e % r);
             float v = (j <= i) ? A[e] : 0.f;
-            if (i == j) v += shift;
+            if (i == j) v = s_diag[i] + shift;
             W[e] = v;
         }
         if (tid == 0) { s_fail = 0; s_dmin = 3.0e38f; s_dmax = 0.f; }

@@ -159,7 +159,8 @@ void qr_stage(const orthdion_plan* p, const Batch& b, const Scratch& sc, Sel in,
             EpStore eg{gram, gram, only_shift ? shift_bit : 0, 1, r, only_shift};
             launch_simt(b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, st);
         }
-        CholArgs ca{gram, linv, r, which, pass, kShiftRel, kCondLimit};
+        CholArgs ca{gram, linv, r, which, pass, kShiftRel, kCondLimit, sel(W_SCRATCH, 0), 0, r};
+        if (tensor) { ca.colsq = sel(W_SCRATCH, sc.ts.colsq); ca.colsq_kb = (int32_t)((rows + 63) / 64); }
         chol_inv_kernel<<<b.count, CH_THREADS, CH_SMEM_BYTES, st>>>(b, ca);
         // dst = src * L^{-T}
         EpStore ea{};
