@@ -120,6 +120,22 @@ int orthdion_get_factors(const orthdion_t* hs, int32_t count, int32_t index, voi
 int orthdion_last_status(const orthdion_t* hs, int32_t count, void* workspace, void* stream,
                          int32_t* flags);
 
+/* Number of kernels this library has launched so far in this process (monotonic). */
+int64_t orthdion_launch_count(void);
+
+/* Optional per-stage timing.  Between profile_begin and profile_end every kernel launch of the
+ * step functions is bracketed by a pair of CUDA events on the launching stream (at most
+ * max_launches launches are recorded; profile_begin creates the events).  profile_end waits for
+ * the recorded events and returns, per stage s < orthdion_stage_count(), the summed device time
+ * ms[s] in milliseconds and the number of launches.  Stages are the kernels of the step: the
+ * packers, Y = B*Q_prev (Alg. 1 line 2), Gram, Cholesky+inverse, apply (the QR of lines 2 and 4),
+ * R = B^T*P (line 3), ColNorm (line 4) and the fused feedback/update pass (lines 5-7).
+ * Not thread-safe; meant for benchmarks. */
+int orthdion_profile_begin(int32_t max_launches);
+int orthdion_profile_end(int32_t n_stages, double* ms, int64_t* launches);
+int32_t orthdion_stage_count(void);
+const char* orthdion_stage_name(int32_t stage);
+
 /* Library/kernels self-description: returns a static string naming the build (arch, engines). */
 const char* orthdion_version(void);
 

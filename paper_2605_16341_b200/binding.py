@@ -77,6 +77,14 @@ def lib() -> ctypes.CDLL:
     L.orthdion_get_factors.argtypes = [pvp, i32, i32, vp, pvp, pvp]
     L.orthdion_last_status.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(i32)]
     L.orthdion_version.restype = ctypes.c_char_p
+    L.orthdion_launch_count.restype = i64
+    L.orthdion_profile_begin.argtypes = [i32]
+    L.orthdion_profile_begin.restype = i32
+    L.orthdion_profile_end.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    L.orthdion_profile_end.restype = i32
+    L.orthdion_stage_count.restype = i32
+    L.orthdion_stage_name.argtypes = [i32]
+    L.orthdion_stage_name.restype = ctypes.c_char_p
     for name in ("create", "destroy", "set_dtypes", "set_lr", "set_scale", "set_ef", "set_engine",
                  "set_passes", "step", "step_grouped", "get_factors", "last_status"):
         getattr(L, "orthdion_" + name).restype = i32
@@ -87,7 +95,9 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ["orthdion_create", "orthdion_destroy", "orthdion_set_dtypes", "orthdion_set_lr",
             "orthdion_set_scale", "orthdion_set_ef", "orthdion_set_engine", "orthdion_set_passes",
             "orthdion_workspace_bytes", "orthdion_workspace_bytes_grouped", "orthdion_step",
-            "orthdion_step_grouped", "orthdion_get_factors", "orthdion_last_status", "orthdion_version"]
+            "orthdion_step_grouped", "orthdion_get_factors", "orthdion_last_status", "orthdion_version",
+            "orthdion_launch_count", "orthdion_profile_begin", "orthdion_profile_end", "orthdion_stage_count",
+            "orthdion_stage_name"]
 
 
 def _check(code, where):
@@ -213,6 +223,23 @@ def orthdion_last_status(hs, workspace, stream=None):
     _check(lib().orthdion_last_status(_harr(hs), len(hs), _dev_ptr(workspace, "workspace"),
                                       _stream_ptr(stream), flags), "orthdion_last_status")
     return list(flags)
+
+
+def orthdion_launch_count() -> int:
+    return lib().orthdion_launch_count()
+
+
+def orthdion_profile_begin(max_launches: int):
+    _check(lib().orthdion_profile_begin(max_launches), "orthdion_profile_begin")
+
+
+def orthdion_profile_end() -> dict:
+    """{stage name: (milliseconds, launches)} for the launches recorded since profile_begin."""
+    n = lib().orthdion_stage_count()
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_int64 * n)()
+    _check(lib().orthdion_profile_end(n, ms, cnt), "orthdion_profile_end")
+    return {lib().orthdion_stage_name(i).decode(): (ms[i], cnt[i]) for i in range(n)}
 
 
 def orthdion_version() -> str:

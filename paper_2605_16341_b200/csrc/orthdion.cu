@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "profile.cuh"
 #include "factor_kernels.cuh"
 #include "simt_kernels.cuh"
 #include "tensor_engine.cuh"
@@ -134,8 +135,10 @@ int ensure_attributes() {
 }
 
 template <class RA, class RB, class EP>
-void launch_simt(const Batch& b, int64_t Md, int64_t Nd, int64_t Kd, RA ra, RB rb, EP ep, cudaStream_t st) {
+void launch_simt(const Batch& b, int64_t Md, int64_t Nd, int64_t Kd, RA ra, RB rb, EP ep, int stage,
+                 cudaStream_t st) {
     dim3 grid((unsigned)((Nd + 63) / 64), (unsigned)((Md + 63) / 64), (unsigned)b.count);
+    prof::Scope scope(stage, st);
     simt_gemm_kernel<RA, RB, EP><<<grid, 256, 0, st>>>(b, Md, Nd, Kd, ra, rb, ep);
 }
 
@@ -157,11 +160,14 @@ void qr_stage(const orthdion_plan* p, const Batch& b, const Scratch& sc, Sel in,
             tensor_gram(p->m, p->n, r, p->passes[1], b, sc.ts, src, rows, gram, only_shift ? shift_bit : 0, st);
         } else {
             EpStore eg{gram, gram, only_shift ? shift_bit : 0, 1, r, only_shift};
-            launch_simt(b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, st);
+            launch_simt(b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, prof::S_GRAM, st);
         }
         CholArgs ca{gram, linv, r, which, pass, kShiftRel, kCondLimit, sel(W_SCRATCH, 0), 0, r};
         if (tensor) { ca.colsq = sel(W_SCRATCH, sc.ts.colsq); ca.colsq_kb = (int32_t)((rows + 63) / 64); }
-        chol_inv_kernel<<<b.count, CH_THREADS, CH_SMEM_BYTES, st>>>(b, ca);
+        {
+            prof::Scope scope(prof::S_CHOL, st);
+            chol_inv_kernel<<<b.count, CH_THREADS, CH_SMEM_BYTES, st>>>(b, ca);
+        }
         // dst = src * L^{-T}
         EpStore ea{};
         if (pass == 1) ea = EpStore{tmpA, tmpA, 0, 1, r, 0};
@@ -170,7 +176,7 @@ void qr_stage(const orthdion_plan* p, const Batch& b, const Scratch& sc, Sel in,
         if (tensor) {
             tensor_apply(p->m, p->n, r, p->passes[1], b, sc.ts, src, rows, linv, ea, st);
         } else {
-            launch_simt(b, rows, r, r, RdPlain{src, r, 1}, RdPlain{linv, r, 1}, ea, st);
+            launch_simt(b, rows, r, r, RdPlain{src, r, 1}, RdPlain{linv, r, 1}, ea, prof::S_APPLY, st);
         }
     }
 }
@@ -185,24 +191,25 @@ void run_batch(const orthdion_plan* p, const Batch& b, const Scratch& sc, cudaSt
 
     // Alg. 1 lines 1-2:  Y = (M + G) Q_prev   -> P slot
     if (tensor) tensor_k1(m, n, r, gb, p->passes[0], b, sc.ts, st);
-    else launch_simt(b, m, r, n, RdBuffer{n, gb, 0}, RdPlain{sQ, 1, r}, EpStore{sP, sP, 0, 0, r, 0}, st);
+    else launch_simt(b, m, r, n, RdBuffer{n, gb, 0}, RdPlain{sQ, 1, r}, EpStore{sP, sP, 0, 0, r, 0}, prof::S_K1, st);
     qr_stage(p, b, sc, sP, m, sP, 0, st);
     // Alg. 1 line 3:  R = (M + G)^T P
     if (tensor) tensor_k3(m, n, r, gb, p->passes[0], b, sc.ts, st);
-    else launch_simt(b, n, r, m, RdBuffer{n, gb, 1}, RdPlain{sP, 1, r}, EpStore{sR, sR, 0, 0, r, 0}, st);
+    else launch_simt(b, n, r, m, RdBuffer{n, gb, 1}, RdPlain{sP, 1, r}, EpStore{sR, sR, 0, 0, r, 0}, prof::S_K3, st);
     // Alg. 1 line 4
     if (p->mode == ORTHDION_MODE_ORTH) {
         qr_stage(p, b, sc, sR, n, sQ, 1, st);
     } else {
         dim3 grid((unsigned)((r + 31) / 32), 1, (unsigned)b.count);
+        prof::Scope scope(prof::S_COLNORM, st);
         colnorm_kernel<<<grid, 1024, 0, st>>>(b, n, r);
     }
     // Alg. 1 lines 5-7:  M <- a B - b P R^T ;  X <- c X - d P Q^T
     if (tensor) {
         tensor_k5(m, n, r, gb, xb, p->passes[2], p->passes[3], p->ef_a, p->ef_b, c, d, b, sc.ts, st);
     } else {
-        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sR, r, 1}, EpErrorFeedback{p->ef_a, p->ef_b, n, gb}, st);
-        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sQ, r, 1}, EpWeights{c, d, n, xb}, st);
+        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sR, r, 1}, EpErrorFeedback{p->ef_a, p->ef_b, n, gb}, prof::S_K5, st);
+        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sQ, r, 1}, EpWeights{c, d, n, xb}, prof::S_K5, st);
     }
 }
 
@@ -339,7 +346,10 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
             w.status = reinterpret_cast<int32_t*>(ws + lay.status_off) + i;
             w.scratch = ws + lay.scratch_off + k * sc.bytes;
         }
-        init_status_kernel<<<1, MAXB, 0, st>>>(*b);
+        {
+            prof::Scope scope(prof::S_MISC, st);
+            init_status_kernel<<<1, MAXB, 0, st>>>(*b);
+        }
         run_batch(p, *b, sc, st);
         cudaError_t ce = cudaGetLastError();
         if (ce != cudaSuccess) {
@@ -382,6 +392,40 @@ int orthdion_last_status(const orthdion_t* hs, int32_t count, void* workspace, v
     CU_CHECK(cudaStreamSynchronize(st));
     return ORTHDION_OK;
 }
+
+int64_t orthdion_launch_count(void) { return prof::g_launches.load(); }
+
+int orthdion_profile_begin(int32_t max_launches) {
+    if (max_launches < 1 || max_launches > (1 << 20)) return ORTHDION_ERR_INVALID_ARG;
+    while (prof::g_pool.size() < (size_t)max_launches * 2) {
+        cudaEvent_t e;
+        CU_CHECK(cudaEventCreate(&e));
+        prof::g_pool.push_back(e);
+    }
+    prof::g_pool_next = 0;
+    prof::g_records.clear();
+    prof::g_enabled = true;
+    return ORTHDION_OK;
+}
+
+int orthdion_profile_end(int32_t n_stages, double* ms, int64_t* launches) {
+    if (!ms || !launches) return ORTHDION_ERR_NULL;
+    if (n_stages < prof::S_COUNT) return ORTHDION_ERR_INVALID_ARG;
+    prof::g_enabled = false;
+    for (int s = 0; s < n_stages; ++s) { ms[s] = 0.0; launches[s] = 0; }
+    for (const prof::Record& rec : prof::g_records) {
+        CU_CHECK(cudaEventSynchronize(rec.end));
+        float t = 0.f;
+        CU_CHECK(cudaEventElapsedTime(&t, rec.beg, rec.end));
+        ms[rec.stage] += t;
+        launches[rec.stage] += 1;
+    }
+    prof::g_records.clear();
+    return ORTHDION_OK;
+}
+
+int32_t orthdion_stage_count(void) { return prof::S_COUNT; }
+const char* orthdion_stage_name(int32_t stage) { return prof::stage_name(stage); }
 
 const char* orthdion_version(void) {
     return "orthdion sm_100a: engines tensor(tcgen05, bf16-split) + simt(fp32)";

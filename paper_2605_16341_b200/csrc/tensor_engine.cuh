@@ -10,6 +10,7 @@
 // stored: transform warps read M and G from HBM, add, split and write the image directly.
 #pragma once
 #include "common.cuh"
+#include "profile.cuh"
 #include "simt_kernels.cuh"
 
 namespace od {
@@ -688,11 +689,12 @@ inline void launch_pack(const Batch& b, Sel src, int64_t rows_s, int64_t cols_s,
     a.src = src; a.rows_s = (int32_t)rows_s; a.cols_s = (int32_t)cols_s; a.trans = trans;
     a.only_if_shifted = shift_bit_only ? 1 : 0; a.shift_bit = shift_bit_only; a.dst = dst;
     dim3 grid((unsigned)dst.kblocks, (unsigned)dst.row_tiles, (unsigned)b.count);
+    prof::Scope scope(prof::S_PACK, st);
     tc::pack_kernel<<<grid, 256, 0, st>>>(b, a);
 }
 
 template <int AMODE, int EPI>
-inline void launch_gemm(const Batch& b, tc::GemmArgs g, cudaStream_t st) {
+inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t st) {
     g.m_tiles = (g.Mrows + tc::BM - 1) / tc::BM;
     g.n_tiles = (g.Ncols + g.BN - 1) / g.BN;
     g.k_blocks = (g.Kdim + tc::BK - 1) / tc::BK;
@@ -701,6 +703,7 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, cudaStream_t st) {
     const int per_sm = std::max<int>(1, (int)((227 * 1024) / smem));
     const int grid = std::min(g.total_tiles, sm_count() * per_sm);
     const int threads = AMODE == tc::A_PACKED ? tc::THREADS_PACKED : tc::THREADS_BUF;
+    prof::Scope scope(stage, st);
     tc::umma_gemm_kernel<AMODE, EPI><<<grid, threads, smem, st>>>(b, g);
 }
 
@@ -714,7 +717,7 @@ inline void tensor_k1(int64_t m, int64_t n, int r, int g_bf16, int passes, const
     g.Mrows = (int32_t)m; g.Ncols = r; g.Kdim = (int32_t)n; g.BN = tensor_bn(r);
     g.passes = passes; g.passes2 = 1; g.g_bf16 = g_bf16; g.ld = n; g.b = qt;
     g.st = EpStore{Sel{W_P, 0, 0}, Sel{W_P, 0, 0}, 0, 0, r, 0};
-    launch_gemm<tc::A_BUF_ROW, tc::EPI_STORE>(b, g, st);
+    launch_gemm<tc::A_BUF_ROW, tc::EPI_STORE>(b, g, prof::S_K1, st);
 }
 
 // R = (M + G)^T P  -> R slot                                      (Alg. 1 line 3)
@@ -727,7 +730,7 @@ inline void tensor_k3(int64_t m, int64_t n, int r, int g_bf16, int passes, const
     g.Mrows = (int32_t)n; g.Ncols = r; g.Kdim = (int32_t)m; g.BN = tensor_bn(r);
     g.passes = passes; g.passes2 = 1; g.g_bf16 = g_bf16; g.ld = n; g.b = pt;
     g.st = EpStore{Sel{W_R, 0, 0}, Sel{W_R, 0, 0}, 0, 0, r, 0};
-    launch_gemm<tc::A_BUF_COL, tc::EPI_STORE>(b, g, st);
+    launch_gemm<tc::A_BUF_COL, tc::EPI_STORE>(b, g, prof::S_K3, st);
 }
 
 // Gram = src^T src (src: rows x r)
@@ -740,7 +743,7 @@ inline void tensor_gram(int64_t, int64_t, int r, int passes, const Batch& b, con
     g.Mrows = r; g.Ncols = r; g.Kdim = (int32_t)rows; g.BN = tensor_bn(r);
     g.passes = passes; g.passes2 = 1; g.a = sp; g.b = sp;
     g.st = EpStore{gram, gram, only_shift_bit, 1, r, only_shift_bit ? 1 : 0};
-    launch_gemm<tc::A_PACKED, tc::EPI_STORE>(b, g, st);
+    launch_gemm<tc::A_PACKED, tc::EPI_STORE>(b, g, prof::S_GRAM, st);
 }
 
 // dst = src * L^{-T}  (src: rows x r, L^{-1} lower triangular r x r)
@@ -756,7 +759,7 @@ inline void tensor_apply(int64_t, int64_t, int r, int passes, const Batch& b, co
     g.Mrows = (int32_t)rows; g.Ncols = r; g.Kdim = r; g.BN = tensor_bn(r);
     g.passes = passes; g.passes2 = 1; g.a = sp; g.b = lp; g.tri = 1;
     g.st = ep;
-    launch_gemm<tc::A_PACKED, tc::EPI_STORE>(b, g, st);
+    launch_gemm<tc::A_PACKED, tc::EPI_STORE>(b, g, prof::S_APPLY, st);
 }
 
 // M <- a (M + G) - b P R^T ;  X <- c X - d P Q^T                  (Alg. 1 lines 5-7)
@@ -774,7 +777,7 @@ inline void tensor_k5(int64_t m, int64_t n, int r, int g_bf16, int x_bf16, int p
     g.passes = passes_m; g.passes2 = passes_x; g.g_bf16 = g_bf16; g.x_bf16 = x_bf16; g.ld = n;
     g.a = pp; g.b = rp; g.b2 = qp;
     g.ef_a = ef_a; g.ef_b = ef_b; g.wc = wc; g.wd = wd;
-    launch_gemm<tc::A_PACKED, tc::EPI_K5>(b, g, st);
+    launch_gemm<tc::A_PACKED, tc::EPI_K5>(b, g, prof::S_K5, st);
 }
 
 }  // namespace od
