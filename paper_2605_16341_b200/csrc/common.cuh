@@ -21,9 +21,11 @@ struct MatWork {
     float* R;           // n x r   (workspace slot)
     int32_t* status;    // one word
     char* scratch;      // per-matrix scratch area
+    int32_t aux0;       // launch-specific per-matrix integer (Cholesky: rows of column-square partials)
+    int32_t aux1;
 };
 
-constexpr int MAXB = 128;   // matrices per launch batch
+constexpr int MAXB = 256;   // matrices per launch batch
 struct Batch {
     int32_t count;
     int32_t pad;
@@ -50,5 +52,49 @@ __device__ __forceinline__ float load_elem(const void* p, int64_t idx, int is_bf
     if (is_bf16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx]);
     return reinterpret_cast<const float*>(p)[idx];
 }
+
+// ---- bf16 splitting ---------------------------------------------------------------------------
+// An fp32 value v is carried through the tensor cores as v = t0 + t1 with t0 = bf16(v),
+// t1 = bf16(v - t0) (round to nearest even): the two terms together hold 16 significand bits.
+
+// two fp32 -> packed bf16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t p) { return __uint_as_float(p << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t p) { return __uint_as_float(p & 0xFFFF0000u); }
+
+// 8 fp32 values -> 16-byte chunk of term 0 and of term 1
+__device__ __forceinline__ void split8(const float (&v)[8], uint4& t0, uint4& t1) {
+    uint32_t a[4], b[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        a[e] = pack_bf16x2(v[2 * e], v[2 * e + 1]);
+        float r0 = v[2 * e] - bf16lo_to_f32(a[e]);
+        float r1 = v[2 * e + 1] - bf16hi_to_f32(a[e]);
+        b[e] = pack_bf16x2(r0, r1);
+    }
+    t0 = make_uint4(a[0], a[1], a[2], a[3]);
+    t1 = make_uint4(b[0], b[1], b[2], b[3]);
+}
+
+// Split image of an fp32 matrix S (rows x cols): the operand format of every tensor-core product.
+// Columns are cut into panels of 64; a panel stores one 128-byte row (64 bf16) per matrix row,
+// rows padded with zeros to a multiple of 128, and the eight 16-byte chunks of a row are
+// XOR-swizzled with (row & 7) (the 128-byte shared-memory swizzle of the MMA descriptors).  Term t
+// of panel p starts at off + (t * panels + p) * rows_pad * 128.  128 consecutive rows of a panel
+// are a K-major operand tile (depth = S columns); 64 consecutive rows of two or more panels are an
+// MN-major operand tile (depth = S rows): bulk copies move either into shared memory unchanged.
+struct ImgRef {
+    int64_t off;        // byte offset in the matrix's scratch area; < 0: absent
+    int32_t rows_pad;   // multiple of 128
+    int32_t panels;     // ceil(cols / 64)
+};
+__device__ __forceinline__ int64_t img_row_offset(const ImgRef& im, int term, int panel, int64_t row) {
+    return im.off + (((int64_t)term * im.panels + panel) * im.rows_pad + row) * 128;
+}
+__device__ __forceinline__ int img_chunk_offset(int row, int chunk) { return ((chunk ^ (row & 7)) << 4); }
 
 }  // namespace od

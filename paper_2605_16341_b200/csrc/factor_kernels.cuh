@@ -71,11 +71,13 @@ struct CholArgs {
     int32_t pass;    // 1, 2 or 3
     float shift_rel; // shift = shift_rel * trace(Gram) on the retry of pass 1
     float cond_limit;// take the shifted path when max diag(L) / min diag(L) exceeds this (pass 1)
-    // Optional fp32 column sums of squares, colsq[kb * colsq_ld + i], kb < colsq_kb: when given they
-    // replace the Gram diagonal.  (The tensor core truncates when it adds into its fp32 accumulator,
-    // which biases long sums of squares low; the off-diagonal sums have no such bias.)
+    // Optional fp32 column sums of squares, colsq[p * r + i] for p < MatWork::aux0 partial rows: when
+    // use_colsq is set they replace the Gram diagonal.  (The tensor core truncates when it adds
+    // into its fp32 accumulator, which biases long sums of squares low; the off-diagonal sums have
+    // no such bias.)
     Sel colsq;
-    int32_t colsq_kb, colsq_ld;
+    int32_t use_colsq, pad;
+    ImgRef img;      // img.off >= 0: also write L^{-1} as a split image (tensor-core operand)
 };
 
 // Factor Gram = L L^T (blocked, right-looking) and overwrite `work` with L^{-1}.
@@ -114,10 +116,10 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         float t = 0.f;
         for (int i = tid; i < r; i += CH_THREADS) {
             float d;
-            if (a.colsq_kb > 0) {
+            if (a.use_colsq) {
                 const float* cs = pick(w, a.colsq);
                 d = 0.f;
-                for (int kb = 0; kb < a.colsq_kb; ++kb) d += cs[(int64_t)kb * a.colsq_ld + i];
+                for (int kb = 0; kb < w.aux0; ++kb) d += cs[(int64_t)kb * r + i];
             } else {
                 d = A[(int64_t)i * r + i];
             }
@@ -326,6 +328,23 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
             }
         }
         __syncthreads();
+    }
+    // ---- split image of L^{-1} for the tensor-core apply product ------------------------------
+    if (a.img.off >= 0) {
+        unsigned char* scr = reinterpret_cast<unsigned char*>(w.scratch);
+        const int chunks = a.img.panels * a.img.rows_pad * 8;
+        for (int q = tid; q < chunks; q += CH_THREADS) {
+            const int c = q % 8, row = (q / 8) % a.img.rows_pad, panel = q / (8 * a.img.rows_pad);
+            const int col = panel * 64 + c * 8;
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = (row < r && col + i < r) ? W[(int64_t)row * r + col + i] : 0.f;
+            uint4 t0, t1;
+            split8(v, t0, t1);
+            const int o = img_chunk_offset(row, c);
+            *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 0, panel, row) + o) = t0;
+            *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 1, panel, row) + o) = t1;
+        }
     }
 }
 

@@ -42,7 +42,8 @@ bool same_class(const orthdion_plan* a, const orthdion_plan* b) {
            a->ef_b == b->ef_b && std::memcmp(a->passes, b->passes, sizeof(a->passes)) == 0;
 }
 
-// Per-matrix scratch carving (byte offsets).  kmax = max(m, n).
+// Per-matrix scratch carving (byte offsets).  gram, linv and the tensor engine's first entries
+// depend on r only, so one Cholesky launch can serve matrices of different shapes.
 struct Scratch {
     int64_t gram, linv, tmpA, tmpB;
     TensorScratch ts;
@@ -52,25 +53,33 @@ struct Scratch {
 Scratch scratch_layout(const orthdion_plan* p) {
     Scratch s{};
     const size_t rr = align_up((size_t)p->r * p->r * 4, 256);
-    const size_t kr = align_up((size_t)std::max(p->m, p->n) * p->r * 4, 256);
     size_t off = 0;
     s.gram = off; off += rr;
     s.linv = off; off += rr;
-    s.tmpA = off; off += kr;
-    s.tmpB = off; off += kr;
-    if (p->engine == ORTHDION_ENGINE_TENSOR) off = tensor_scratch_layout(p->m, p->n, p->r, off, &s.ts);
-    s.bytes = align_up(off, 256);
+    if (p->engine == ORTHDION_ENGINE_TENSOR) {
+        off = tensor_scratch_layout(p->m, p->n, p->r, off, &s.ts);
+    } else {
+        const size_t kr = align_up((size_t)std::max(p->m, p->n) * p->r * 4, 256);
+        s.tmpA = off; off += kr;
+        s.tmpB = off; off += kr;
+    }
+    s.bytes = align_up(off, 1024);
     return s;
 }
 
+// A launch batch: matrices of one class.  A group: batches that are stepped together, stage by
+// stage, so that the short serial kernels (the r x r Cholesky) of all of them run side by side.
 struct Batching {
-    std::vector<std::vector<int>> batches;   // matrix indices per launch batch, class by class
-    size_t scratch_bytes = 0;                // max over batches
+    std::vector<std::vector<int>> batches;   // matrix indices per launch batch
+    std::vector<std::vector<int>> groups;    // batch indices per group
+    std::vector<size_t> batch_off;           // scratch offset of each batch inside its group
+    size_t scratch_bytes = 0;                // max over groups
 };
 
 Batching make_batches(const orthdion_t* hs, int32_t count) {
     Batching out;
     std::vector<char> done(count, 0);
+    size_t group_bytes = 0;
     for (int i = 0; i < count; ++i) {
         if (done[i]) continue;
         std::vector<int> cls;
@@ -83,14 +92,22 @@ Batching make_batches(const orthdion_t* hs, int32_t count) {
         const size_t bs = (cls.size() + nb - 1) / nb;
         for (size_t b = 0; b < cls.size(); b += bs) {
             std::vector<int> one(cls.begin() + b, cls.begin() + std::min(cls.size(), b + bs));
-            out.scratch_bytes = std::max(out.scratch_bytes, one.size() * per);
+            const size_t bytes = one.size() * per;
+            if (out.groups.empty() || group_bytes + bytes > kScratchBudget) {
+                out.groups.emplace_back();
+                group_bytes = 0;
+            }
+            out.groups.back().push_back((int)out.batches.size());
+            out.batch_off.push_back(group_bytes);
+            group_bytes += bytes;
+            out.scratch_bytes = std::max(out.scratch_bytes, group_bytes);
             out.batches.push_back(std::move(one));
         }
     }
     return out;
 }
 
-// Workspace: [status words][P_0 R_0][P_1 R_1]...[scratch of the largest batch]
+// Workspace: [status words][P_0 R_0][P_1 R_1]...[scratch of the largest group]
 struct Layout {
     std::vector<size_t> p_off, r_off;
     size_t status_off = 0, scratch_off = 0, total = 0;
@@ -105,8 +122,8 @@ Layout make_layout(const orthdion_t* hs, int32_t count, size_t scratch_bytes) {
         l.p_off[i] = off; off += align_up((size_t)hs[i]->m * hs[i]->r * 4, 256);
         l.r_off[i] = off; off += align_up((size_t)hs[i]->n * hs[i]->r * 4, 256);
     }
-    l.scratch_off = off;
-    l.total = off + scratch_bytes;
+    l.scratch_off = align_up(off, 1024);
+    l.total = l.scratch_off + scratch_bytes;
     return l;
 }
 
@@ -144,72 +161,167 @@ void launch_simt(const Batch& b, int64_t Md, int64_t Nd, int64_t Kd, RA ra, RB r
 
 Sel sel(int where, int64_t off = 0) { return Sel{where, 0, off}; }
 
-// ---- tall-skinny QR of `in` (rows x r) into `fin` (CholeskyQR2; third pass when flagged) -------
-void qr_stage(const orthdion_plan* p, const Batch& b, const Scratch& sc, Sel in, int64_t rows, Sel fin,
-              int which, cudaStream_t st) {
-    const int r = p->r;
-    const int shift_bit = which ? ST_SHIFT_R : ST_SHIFT_L;
-    const Sel gram = sel(W_SCRATCH, sc.gram), linv = sel(W_SCRATCH, sc.linv);
-    const Sel tmpA = sel(W_SCRATCH, sc.tmpA), tmpB = sel(W_SCRATCH, sc.tmpB);
-    const bool tensor = p->engine == ORTHDION_ENGINE_TENSOR;
-    for (int pass = 1; pass <= 3; ++pass) {
-        const Sel src = pass == 1 ? in : (pass == 2 ? tmpA : tmpB);
-        const int only_shift = pass == 3;
-        // Gram = src^T src
-        if (tensor) {
-            tensor_gram(p->m, p->n, r, p->passes[1], b, sc.ts, src, rows, gram, only_shift ? shift_bit : 0, st);
-        } else {
-            EpStore eg{gram, gram, only_shift ? shift_bit : 0, 1, r, only_shift};
-            launch_simt(b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, prof::S_GRAM, st);
+// One class of a group while it is being stepped.
+struct ClassRun {
+    const orthdion_plan* p;
+    Batch* b;
+    Scratch sc;
+    bool tensor() const { return p->engine == ORTHDION_ENGINE_TENSOR; }
+};
+
+// Cholesky + inverse of every class's Gram matrix: classes of equal (r, engine) share launches.
+void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int which, int pass,
+                Batch* merged, cudaStream_t st) {
+    std::vector<char> done(which_cls.size(), 0);
+    for (size_t i = 0; i < which_cls.size(); ++i) {
+        if (done[i]) continue;
+        const ClassRun& lead = cls[which_cls[i]];
+        const int r = lead.p->r;
+        CholArgs ca{};
+        ca.gram = sel(W_SCRATCH, lead.sc.gram); ca.work = sel(W_SCRATCH, lead.sc.linv);
+        ca.r = r; ca.which = which; ca.pass = pass; ca.shift_rel = kShiftRel; ca.cond_limit = kCondLimit;
+        ca.colsq = sel(W_SCRATCH, 0); ca.use_colsq = 0; ca.img = no_img();
+        if (lead.tensor()) {
+            ca.colsq = sel(W_SCRATCH, lead.sc.ts.colsq); ca.use_colsq = 1; ca.img = lead.sc.ts.linv;
         }
-        CholArgs ca{gram, linv, r, which, pass, kShiftRel, kCondLimit, sel(W_SCRATCH, 0), 0, r};
-        if (tensor) { ca.colsq = sel(W_SCRATCH, sc.ts.colsq); ca.colsq_kb = (int32_t)((rows + 63) / 64); }
-        {
+        merged->count = 0; merged->pad = 0;
+        auto flush = [&]() {
+            if (!merged->count) return;
             prof::Scope scope(prof::S_CHOL, st);
-            chol_inv_kernel<<<b.count, CH_THREADS, CH_SMEM_BYTES, st>>>(b, ca);
+            chol_inv_kernel<<<merged->count, CH_THREADS, CH_SMEM_BYTES, st>>>(*merged, ca);
+            merged->count = 0;
+        };
+        for (size_t j = i; j < which_cls.size(); ++j) {
+            const ClassRun& c = cls[which_cls[j]];
+            if (done[j] || c.p->r != r || c.tensor() != lead.tensor()) continue;
+            done[j] = 1;
+            const int64_t rows = which ? c.p->n : c.p->m;
+            for (int k = 0; k < c.b->count; ++k) {
+                MatWork& w = merged->w[merged->count++];
+                w = c.b->w[k];
+                w.aux0 = (int32_t)(4 * ((rows + 127) / 128));
+                if (merged->count == MAXB) flush();
+            }
         }
-        // dst = src * L^{-T}
-        EpStore ea{};
-        if (pass == 1) ea = EpStore{tmpA, tmpA, 0, 1, r, 0};
-        else if (pass == 2) ea = EpStore{fin, tmpB, shift_bit, 1, r, 0};
-        else ea = EpStore{fin, fin, shift_bit, 1, r, 1};
-        if (tensor) {
-            tensor_apply(p->m, p->n, r, p->passes[1], b, sc.ts, src, rows, linv, ea, st);
-        } else {
-            launch_simt(b, rows, r, r, RdPlain{src, r, 1}, RdPlain{linv, r, 1}, ea, prof::S_APPLY, st);
+        flush();
+    }
+}
+
+// ---- tall-skinny QR of every class in `which_cls` (CholeskyQR2; third pass when flagged) --------
+// which = 0: P = orth(Y) (Alg. 1 line 2), which = 1: Q = orth(R) (Alg. 1 line 4).
+// Tensor engine: the input is an image (w0 holds Y, image r holds R); SIMT engine: fp32 slots.
+void qr_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int which, Batch* merged,
+              cudaStream_t st) {
+    const int shift_bit = which ? ST_SHIFT_R : ST_SHIFT_L;
+    for (int pass = 1; pass <= 3; ++pass) {
+        const int only_shift = pass == 3;
+        for (int ci : which_cls) {
+            ClassRun& c = cls[ci];
+            const int r = c.p->r;
+            const int64_t rows = which ? c.p->n : c.p->m;
+            const Sel gram = sel(W_SCRATCH, c.sc.gram);
+            if (c.tensor()) {
+                const TensorScratch& ts = c.sc.ts;
+                const ImgRef in = which ? ts.r : img_view(ts.w0, rows);
+                const ImgRef src = pass == 1 ? in : (pass == 2 ? img_view(ts.w1, rows) : img_view(ts.w0, rows));
+                tensor_gram(r, c.p->passes[1], *c.b, src, rows, gram, only_shift ? shift_bit : 0, st);
+            } else {
+                const Sel in = which ? sel(W_R) : sel(W_P);
+                const Sel src = pass == 1 ? in : (pass == 2 ? sel(W_SCRATCH, c.sc.tmpA) : sel(W_SCRATCH, c.sc.tmpB));
+                EpStore eg{gram, gram, only_shift ? shift_bit : 0, 1, r, only_shift};
+                launch_simt(*c.b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, prof::S_GRAM, st);
+            }
+        }
+        chol_stage(cls, which_cls, which, pass, merged, st);
+        for (int ci : which_cls) {
+            ClassRun& c = cls[ci];
+            const int r = c.p->r;
+            const int64_t rows = which ? c.p->n : c.p->m;
+            const Sel fin = which ? sel(W_Q) : sel(W_P);
+            if (c.tensor()) {
+                const TensorScratch& ts = c.sc.ts;
+                const ImgRef in = which ? ts.r : img_view(ts.w0, rows);
+                const ImgRef w0 = img_view(ts.w0, rows), w1 = img_view(ts.w1, rows);
+                const ImgRef src = pass == 1 ? in : (pass == 2 ? w1 : w0);
+                tc::Dest to_fin = dest_none();
+                to_fin.f32 = fin; to_fin.has_f32 = 1; to_fin.img = which ? ts.q : ts.p;
+                tc::Dest to_w1 = dest_none(); to_w1.img = w1; to_w1.colsq = 1;
+                tc::Dest to_w0 = dest_none(); to_w0.img = w0; to_w0.colsq = 1;
+                tc::OutSpec out{};
+                out.ld = r; out.shift_bit = 0; out.only_if_shifted = 0;
+                if (pass == 1) { out.normal = to_w1; out.shifted = to_w1; }
+                else if (pass == 2) { out.normal = to_fin; out.shifted = to_w0; out.shift_bit = shift_bit; }
+                else { out.normal = to_fin; out.shifted = to_fin; out.shift_bit = shift_bit; out.only_if_shifted = 1; }
+                tensor_apply(r, c.p->passes[1], *c.b, ts, src, rows, out, st);
+            } else {
+                const Sel in = which ? sel(W_R) : sel(W_P);
+                const Sel tmpA = sel(W_SCRATCH, c.sc.tmpA), tmpB = sel(W_SCRATCH, c.sc.tmpB);
+                const Sel linv = sel(W_SCRATCH, c.sc.linv);
+                const Sel src = pass == 1 ? in : (pass == 2 ? tmpA : tmpB);
+                EpStore ea{};
+                if (pass == 1) ea = EpStore{tmpA, tmpA, 0, 1, r, 0};
+                else if (pass == 2) ea = EpStore{fin, tmpB, shift_bit, 1, r, 0};
+                else ea = EpStore{fin, fin, shift_bit, 1, r, 1};
+                launch_simt(*c.b, rows, r, r, RdPlain{src, r, 1}, RdPlain{linv, r, 1}, ea, prof::S_APPLY, st);
+            }
         }
     }
 }
 
-void run_batch(const orthdion_plan* p, const Batch& b, const Scratch& sc, cudaStream_t st) {
-    const int64_t m = p->m, n = p->n;
-    const int r = p->r;
-    const int gb = p->g_dtype == ORTHDION_DTYPE_BF16, xb = p->x_dtype == ORTHDION_DTYPE_BF16;
-    const bool tensor = p->engine == ORTHDION_ENGINE_TENSOR;
-    const float c = 1.f - p->eta * p->wd, d = p->eta * p->scale;
+// One step of every class of a group, stage by stage.
+void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
     const Sel sP = sel(W_P), sR = sel(W_R), sQ = sel(W_Q);
-
-    // Alg. 1 lines 1-2:  Y = (M + G) Q_prev   -> P slot
-    if (tensor) tensor_k1(m, n, r, gb, p->passes[0], b, sc.ts, st);
-    else launch_simt(b, m, r, n, RdBuffer{n, gb, 0}, RdPlain{sQ, 1, r}, EpStore{sP, sP, 0, 0, r, 0}, prof::S_K1, st);
-    qr_stage(p, b, sc, sP, m, sP, 0, st);
+    std::vector<int> all, orth;
+    for (size_t i = 0; i < cls.size(); ++i) {
+        all.push_back((int)i);
+        if (cls[i].p->mode == ORTHDION_MODE_ORTH) orth.push_back((int)i);
+    }
+    for (ClassRun& c : cls) {
+        prof::Scope scope(prof::S_MISC, st);
+        init_status_kernel<<<(c.b->count + 255) / 256, 256, 0, st>>>(*c.b);
+    }
+    // Alg. 1 lines 1-2:  Y = (M + G) Q_prev
+    for (ClassRun& c : cls) {
+        const orthdion_plan* p = c.p;
+        const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
+        if (c.tensor()) tensor_k1(p->m, p->n, p->r, gb, p->passes[0], *c.b, c.sc.ts, st);
+        else launch_simt(*c.b, p->m, p->r, p->n, RdBuffer{p->n, gb, 0}, RdPlain{sQ, 1, p->r},
+                         EpStore{sP, sP, 0, 0, p->r, 0}, prof::S_K1, st);
+    }
+    qr_stage(cls, all, 0, merged, st);
     // Alg. 1 line 3:  R = (M + G)^T P
-    if (tensor) tensor_k3(m, n, r, gb, p->passes[0], b, sc.ts, st);
-    else launch_simt(b, n, r, m, RdBuffer{n, gb, 1}, RdPlain{sP, 1, r}, EpStore{sR, sR, 0, 0, r, 0}, prof::S_K3, st);
+    for (ClassRun& c : cls) {
+        const orthdion_plan* p = c.p;
+        const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
+        if (c.tensor()) tensor_k3(p->m, p->n, p->r, gb, p->passes[0], *c.b, c.sc.ts, st);
+        else launch_simt(*c.b, p->n, p->r, p->m, RdBuffer{p->n, gb, 1}, RdPlain{sP, 1, p->r},
+                         EpStore{sR, sR, 0, 0, p->r, 0}, prof::S_K3, st);
+    }
     // Alg. 1 line 4
-    if (p->mode == ORTHDION_MODE_ORTH) {
-        qr_stage(p, b, sc, sR, n, sQ, 1, st);
-    } else {
-        dim3 grid((unsigned)((r + 31) / 32), 1, (unsigned)b.count);
-        prof::Scope scope(prof::S_COLNORM, st);
-        colnorm_kernel<<<grid, 1024, 0, st>>>(b, n, r);
+    qr_stage(cls, orth, 1, merged, st);
+    for (ClassRun& c : cls) {
+        const orthdion_plan* p = c.p;
+        if (p->mode == ORTHDION_MODE_ORTH) continue;
+        {
+            dim3 grid((unsigned)((p->r + 31) / 32), 1, (unsigned)c.b->count);
+            prof::Scope scope(prof::S_COLNORM, st);
+            colnorm_kernel<<<grid, 1024, 0, st>>>(*c.b, p->n, p->r);
+        }
+        if (c.tensor()) launch_pack(*c.b, sQ, p->n, p->r, c.sc.ts.q, st);
     }
     // Alg. 1 lines 5-7:  M <- a B - b P R^T ;  X <- c X - d P Q^T
-    if (tensor) {
-        tensor_k5(m, n, r, gb, xb, p->passes[2], p->passes[3], p->ef_a, p->ef_b, c, d, b, sc.ts, st);
-    } else {
-        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sR, r, 1}, EpErrorFeedback{p->ef_a, p->ef_b, n, gb}, prof::S_K5, st);
-        launch_simt(b, m, n, r, RdPlain{sP, r, 1}, RdPlain{sQ, r, 1}, EpWeights{c, d, n, xb}, prof::S_K5, st);
+    for (ClassRun& c : cls) {
+        const orthdion_plan* p = c.p;
+        const int gb = p->g_dtype == ORTHDION_DTYPE_BF16, xb = p->x_dtype == ORTHDION_DTYPE_BF16;
+        const float cc = 1.f - p->eta * p->wd, dd = p->eta * p->scale;
+        if (c.tensor()) {
+            tensor_k5(p->m, p->n, p->r, gb, xb, p->passes[2], p->passes[3], p->ef_a, p->ef_b, cc, dd, *c.b, c.sc.ts, st);
+        } else {
+            launch_simt(*c.b, p->m, p->n, p->r, RdPlain{sP, p->r, 1}, RdPlain{sR, p->r, 1},
+                        EpErrorFeedback{p->ef_a, p->ef_b, p->n, gb}, prof::S_K5, st);
+            launch_simt(*c.b, p->m, p->n, p->r, RdPlain{sP, p->r, 1}, RdPlain{sQ, p->r, 1},
+                        EpWeights{cc, dd, p->n, xb}, prof::S_K5, st);
+        }
     }
 }
 
@@ -330,27 +442,29 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     char* ws = reinterpret_cast<char*>(workspace);
-    Batch* b = new Batch();
+    std::vector<Batch> pool(bt.batches.size() + 1);
+    Batch* merged = &pool[bt.batches.size()];
     int rc = ORTHDION_OK;
-    for (const auto& idx : bt.batches) {
-        const orthdion_plan* p = hs[idx[0]];
-        const Scratch sc = scratch_layout(p);
-        b->count = (int32_t)idx.size();
-        b->pad = 0;
-        for (size_t k = 0; k < idx.size(); ++k) {
-            const int i = idx[k];
-            MatWork& w = b->w[k];
-            w.X = X[i]; w.M = M[i]; w.G = G[i]; w.Q = Q[i];
-            w.P = reinterpret_cast<float*>(ws + lay.p_off[i]);
-            w.R = reinterpret_cast<float*>(ws + lay.r_off[i]);
-            w.status = reinterpret_cast<int32_t*>(ws + lay.status_off) + i;
-            w.scratch = ws + lay.scratch_off + k * sc.bytes;
+    for (const auto& grp : bt.groups) {
+        std::vector<ClassRun> cls;
+        for (int bi : grp) {
+            const auto& idx = bt.batches[bi];
+            ClassRun c{hs[idx[0]], &pool[bi], scratch_layout(hs[idx[0]])};
+            c.b->count = (int32_t)idx.size();
+            c.b->pad = 0;
+            for (size_t k = 0; k < idx.size(); ++k) {
+                const int i = idx[k];
+                MatWork& w = c.b->w[k];
+                w.X = X[i]; w.M = M[i]; w.G = G[i]; w.Q = Q[i];
+                w.P = reinterpret_cast<float*>(ws + lay.p_off[i]);
+                w.R = reinterpret_cast<float*>(ws + lay.r_off[i]);
+                w.status = reinterpret_cast<int32_t*>(ws + lay.status_off) + i;
+                w.scratch = ws + lay.scratch_off + bt.batch_off[bi] + k * c.sc.bytes;
+                w.aux0 = 0; w.aux1 = 0;
+            }
+            cls.push_back(c);
         }
-        {
-            prof::Scope scope(prof::S_MISC, st);
-            init_status_kernel<<<1, MAXB, 0, st>>>(*b);
-        }
-        run_batch(p, *b, sc, st);
+        run_group(cls, merged, st);
         cudaError_t ce = cudaGetLastError();
         if (ce != cudaSuccess) {
             std::fprintf(stderr, "orthdion: launch failed: %s\n", cudaGetErrorString(ce));
@@ -358,7 +472,6 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
             break;
         }
     }
-    delete b;
     return rc;
 }
 

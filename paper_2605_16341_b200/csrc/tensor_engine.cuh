@@ -1,14 +1,22 @@
 // Tensor-core engine: tcgen05 (5th-generation tensor core) kernels with accumulators in tensor
 // memory.  Every matrix product of the step is a sum of bf16 products with fp32 accumulation:
-// an fp32 operand v is split as v = t0 + t1 (+ ...) with t0 = bf16(v), t1 = bf16(v - t0), and
-// "3 passes" means t0*u0 + t0*u1 + t1*u0 (relative error about 2^-16), "1 pass" t0*u0.
+// an fp32 operand v is split as v = t0 + t1 with t0 = bf16(v), t1 = bf16(v - t0), and "3 passes"
+// means t0*u0 + t0*u1 + t1*u0 (relative error about 2^-16), "1 pass" t0*u0.
 //
-// Operand staging.  Small operands (Q, P, R, L^{-1} and the QR intermediates) are first written by
-// pack kernels as ready-made shared-memory images (128-row x 64-deep bf16 tiles, 128-byte rows,
-// 16-byte chunks XOR-swizzled by row) and fetched with bulk asynchronous copies (TMA engine,
-// cp.async.bulk) that complete on an mbarrier.  The big operand B = M + G (Alg. 1 line 1) is never
-// stored: transform warps read M and G from HBM, add, split and write the image directly.
+// Operands.  Every small operand (Q, Y, P, R, L^{-1} and the QR intermediates) lives in global
+// memory as a split image (common.cuh): ready-made swizzled shared-memory tiles that bulk
+// asynchronous copies (TMA engine, cp.async.bulk) drop into an operand ring, usable both K-major
+// and MN-major, so no kernel ever transposes.  Images are written by the epilogue of the kernel
+// that produces the matrix; only Q_prev (caller-owned fp32) is packed by a kernel of its own.
+// The big operand B = M + G (Alg. 1 line 1) is never stored: transform warps read M and G from
+// HBM, add, split and write the A tile directly.
+//
+// One CTA per SM walks a tile list.  Two rings in shared memory: A tiles of 128 x 64 (both terms,
+// 32 KB) and N-side pieces (a slice of the other operand, at most 48 KB), each with full/empty
+// mbarriers; accumulators (up to 128 x 512 fp32) sit in tensor memory.
 #pragma once
+#include <algorithm>
+
 #include "common.cuh"
 #include "profile.cuh"
 #include "simt_kernels.cuh"
@@ -16,35 +24,57 @@
 namespace od {
 namespace tc {
 
-constexpr int BM = 128;              // tile rows (MMA M)
-constexpr int BK = 64;               // depth of one stage: 64 bf16 = one 128-byte swizzled row
-constexpr int TILE_BYTES = 128 * 128;   // one 128 x 64 bf16 image
-constexpr int STAGES = 2;
-constexpr int NUM_EPI_WARPS = 4;
-constexpr int NUM_XF_WARPS = 8;
-constexpr int THREADS_PACKED = 32 * (2 + NUM_EPI_WARPS);
-constexpr int THREADS_BUF = 32 * (2 + NUM_EPI_WARPS + NUM_XF_WARPS);
+constexpr int BM = 128;                      // tile rows (MMA M)
+constexpr int BK = 64;                       // depth of one A tile: 64 bf16 = one 128-byte row
+constexpr int A_TERM_BYTES = 128 * 128;      // one 128 x 64 bf16 tile
+constexpr int A_SLOT_BYTES = 2 * A_TERM_BYTES;
+constexpr int A_SLOTS = 2;
+constexpr int MAX_N_SLOTS = 6;
+constexpr int NUM_XF_WARPS = 16;             // transform warps of the kernels that form B = M + G
+constexpr int STAGING_BYTES_PER_WARP = 8192; // K5 epilogue: two 32 x 32 fp32 blocks per warp
+constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 
-enum AMode : int { A_PACKED = 0, A_BUF_ROW = 1, A_BUF_COL = 2 };
+enum AMode : int { A_IMG_K = 0, A_IMG_MN = 1, A_BUF_ROW = 2, A_BUF_COL = 3 };
+enum NMode : int { N_IMG_K = 0, N_IMG_MN = 1 };
 enum EpiMode : int { EPI_STORE = 0, EPI_K5 = 1 };
 
-// A packed operand inside a matrix's scratch area.  Tile (kb, term, row_tile) lives at
-// off + ((kb * terms + term) * row_tiles + row_tile) * TILE_BYTES.
-struct PackRef {
-    int64_t off;
-    int32_t row_tiles, terms, kblocks, pad;
+__host__ __device__ constexpr int epi_warps(int epi) { return epi == EPI_K5 ? 8 : 4; }
+__host__ __device__ constexpr bool a_is_buf(int amode) { return amode == A_BUF_ROW || amode == A_BUF_COL; }
+__host__ __device__ constexpr int gemm_threads(int amode, int epi) {
+    return 32 * (2 + epi_warps(epi) + (a_is_buf(amode) ? NUM_XF_WARPS : 0));
+}
+
+// Where the result of an EPI_STORE product goes.
+struct Dest {
+    Sel f32;            // fp32 row-major copy (leading dimension OutSpec::ld) when has_f32
+    ImgRef img;         // split image when img.off >= 0
+    int32_t has_f32;
+    int32_t colsq;      // also write per-(32-row block) column sums of squares (fp32)
+};
+struct OutSpec {
+    Dest normal, shifted;      // `shifted` is used when the matrix's status has shift_bit set
+    int32_t shift_bit;
+    int32_t only_if_shifted;   // skip the matrix unless shift_bit is set
+    int64_t ld;
 };
 
 struct GemmArgs {
-    int32_t Mrows, Ncols, Kdim, BN;
-    int32_t m_tiles, n_tiles, k_blocks, tri;
-    int32_t passes, passes2, total_tiles, g_bf16;
-    int32_t x_bf16, pad0;
-    int64_t ld;
-    PackRef a, b, b2;
+    int32_t Mrows, Ncols, Kdim, BN;          // BN: nominal tile width (multiple of 16, <= 512)
+    int32_t m_tiles, n_tiles, k_blocks, total_tiles;
+    int32_t tri;                             // N-side is lower triangular (apply): skip depth beyond the tile
+    int32_t lower_only;                      // symmetric result (Gram): skip tiles above the diagonal
+    int32_t passes, passes2;                 // 1 or 3; passes2: second product of the fused pass
+    int32_t ks;                              // N_IMG_MN: depth of one N-side piece (16, 32 or 64)
+    int32_t n_slots, n_piece_bytes;          // N ring
+    int32_t acc_bufs;                        // accumulator buffers in tensor memory (1 or 2)
+    int32_t tmem_cols;                       // allocation (power of two >= 32)
+    int32_t pad0;
+    int64_t ld;                              // leading dimension of M, G, X
+    ImgRef a, n1, n2;
+    int64_t colsq_off;                       // scratch offset of the column-square partials
     float ef_a, ef_b, wc, wd;
-    EpStore st;
+    OutSpec out;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -135,33 +165,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)2 << 61;     // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = n; a_mn = 1 for an MN-major A.
-__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t a_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | ((n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-// ---- bf16 splitting -----------------------------------------------------------------------------
-// two fp32 -> packed bf16x2 (lo in the low half), round to nearest even
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ float bf16lo_to_f32(uint32_t p) { return __uint_as_float(p << 16); }
-__device__ __forceinline__ float bf16hi_to_f32(uint32_t p) { return __uint_as_float(p & 0xFFFF0000u); }
-
-// 8 fp32 values -> chunk of term 0 and chunk of term 1 (each 8 bf16 = 16 bytes)
-__device__ __forceinline__ void split8(const float (&v)[8], uint4& t0, uint4& t1) {
-    uint32_t a[4], b[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        a[e] = pack_bf16x2(v[2 * e], v[2 * e + 1]);
-        float r0 = v[2 * e] - bf16lo_to_f32(a[e]);
-        float r1 = v[2 * e + 1] - bf16hi_to_f32(a[e]);
-        b[e] = pack_bf16x2(r0, r1);
-    }
-    t0 = make_uint4(a[0], a[1], a[2], a[3]);
-    t1 = make_uint4(b[0], b[1], b[2], b[3]);
+// Instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = n; a_mn / b_mn = 1 for an
+// MN-major A / B operand (0: K-major).
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t a_mn, uint32_t b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) | ((n >> 3) << 17) |
+           ((uint32_t)(BM >> 4) << 24);
 }
 
 __device__ __forceinline__ void load8(const void* base, int64_t idx, int is_bf16, float (&v)[8]) {
@@ -180,95 +188,47 @@ __device__ __forceinline__ void load8(const void* base, int64_t idx, int is_bf16
 }
 
 // ------------------------------------------------------------------------------------------
-// Pack kernel: fp32 matrix S (rows_s x cols_s, row-major, leading dimension cols_s) -> packed operand.
-//   trans = 0: operand row = S row,    depth = S column
-//   trans = 1: operand row = S column, depth = S row
-// One CTA per 128 x 64 tile (all terms), 256 threads.
+// Pack kernel: fp32 matrix S (rows x cols, row-major, cols % 8 == 0) -> split image.
+// One CTA per (panel, 128-row block), 256 threads; rows beyond `rows` are written as zeros.
 // ------------------------------------------------------------------------------------------
 struct PackArgs {
     Sel src;
-    int32_t rows_s, cols_s;
-    int32_t trans, only_if_shifted, shift_bit, colsq_ld;
-    int64_t colsq_off;   // >= 0 (trans only): also write fp32 column sums of squares of this 64-row block
-    PackRef dst;
+    int32_t rows, cols;
+    ImgRef dst;
 };
 
 __global__ void __launch_bounds__(256)
 pack_kernel(const __grid_constant__ Batch batch, PackArgs a) {
     const MatWork& w = batch.w[blockIdx.z];
-    const int st = *w.status;
-    if (st & ST_FAILED) return;
-    if (a.only_if_shifted && !(st & a.shift_bit)) return;
+    if (*w.status & ST_FAILED) return;
     const float* S = pick(w, a.src);
-    const int rt = blockIdx.y, kb = blockIdx.x;
-    unsigned char* out0 = reinterpret_cast<unsigned char*>(w.scratch + a.dst.off) +
-                          ((int64_t)(kb * a.dst.terms + 0) * a.dst.row_tiles + rt) * TILE_BYTES;
-    unsigned char* out1 = out0 + (int64_t)a.dst.row_tiles * TILE_BYTES;
-    const int tid = threadIdx.x;
-    if (!a.trans) {
+    const int panel = blockIdx.x, rb = blockIdx.y;
+    unsigned char* out0 = reinterpret_cast<unsigned char*>(w.scratch) + img_row_offset(a.dst, 0, panel, (int64_t)rb * 128);
+    unsigned char* out1 = reinterpret_cast<unsigned char*>(w.scratch) + img_row_offset(a.dst, 1, panel, (int64_t)rb * 128);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int q = tid + 256 * e;
-            const int rho = q / 8, c = q % 8;
-            const int64_t gr = (int64_t)rt * 128 + rho, gk = (int64_t)kb * 64 + c * 8;
-            float v[8];
-            if (gr < a.rows_s && gk < a.cols_s) {   // cols_s % 8 == 0
-                load8(S, gr * a.cols_s + gk, 0, v);
-            } else {
+    for (int e = 0; e < 4; ++e) {
+        const int q = threadIdx.x + 256 * e;
+        const int rho = q / 8, c = q % 8;
+        const int64_t gr = (int64_t)rb * 128 + rho, gk = (int64_t)panel * 64 + c * 8;
+        float v[8];
+        if (gr < a.rows && gk < a.cols) {
+            load8(S, gr * a.cols + gk, 0, v);
+        } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = 0.f;
-            }
-            uint4 t0, t1;
-            split8(v, t0, t1);
-            const int o = rho * 128 + ((c ^ (rho & 7)) << 4);
-            *reinterpret_cast<uint4*>(out0 + o) = t0;
-            if (a.dst.terms > 1) *reinterpret_cast<uint4*>(out1 + o) = t1;
+            for (int i = 0; i < 8; ++i) v[i] = 0.f;
         }
-    } else {
-        __shared__ float tile[64][129];
-        // S rows kb*64 .. +63 (depth), S cols rt*128 .. +127 (operand rows)
-        for (int e = tid; e < 64 * 32; e += 256) {
-            const int kk = e / 32, c4 = e % 32;
-            const int64_t gk = (int64_t)kb * 64 + kk, gc = (int64_t)rt * 128 + c4 * 4;
-            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (gk < a.rows_s && gc < a.cols_s)     // cols_s % 4 == 0
-                x = *reinterpret_cast<const float4*>(S + gk * a.cols_s + gc);
-            tile[kk][c4 * 4 + 0] = x.x; tile[kk][c4 * 4 + 1] = x.y;
-            tile[kk][c4 * 4 + 2] = x.z; tile[kk][c4 * 4 + 3] = x.w;
-        }
-        __syncthreads();
-        if (a.colsq_off >= 0 && tid < 128 && rt * 128 + tid < a.cols_s) {
-            float s = 0.f;
-#pragma unroll 8
-            for (int kk = 0; kk < 64; ++kk) s = fmaf(tile[kk][tid], tile[kk][tid], s);
-            reinterpret_cast<float*>(w.scratch + a.colsq_off)[(int64_t)kb * a.colsq_ld + rt * 128 + tid] = s;
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int q = tid + 256 * e;
-            const int rho = q % 128, c = q / 128;
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = tile[c * 8 + i][rho];
-            uint4 t0, t1;
-            split8(v, t0, t1);
-            const int o = rho * 128 + ((c ^ (rho & 7)) << 4);
-            *reinterpret_cast<uint4*>(out0 + o) = t0;
-            if (a.dst.terms > 1) *reinterpret_cast<uint4*>(out1 + o) = t1;
-        }
+        uint4 t0, t1;
+        split8(v, t0, t1);
+        const int o = rho * 128 + img_chunk_offset(rho, c);
+        *reinterpret_cast<uint4*>(out0 + o) = t0;
+        *reinterpret_cast<uint4*>(out1 + o) = t1;
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// The GEMM kernel.  Persistent CTAs walk the tile list t = blockIdx.x, blockIdx.x + gridDim.x, ...
-//   warp 0      bulk-copy producer (packed operands)
-//   warp 1      MMA issuer, owns the tensor-memory allocation
-//   warps 2-5   epilogue (tensor memory -> registers -> global)
-//   warps 6-13  transform warps (A_BUF_* only): form B = M + G, split, write the A image
-// Accumulators are double-buffered in tensor memory so that the epilogue of tile i overlaps the
-// main loop of tile i+1.
+// Tile bookkeeping shared by all roles of the GEMM kernel
 // ------------------------------------------------------------------------------------------
-struct TileCoord { int b, mt, nt, kb_end; bool active; };
+struct TileCoord { int b, mt, nt, n0, bn, kb_end; bool active; };
 
 template <int EPI>
 __device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmArgs& g, int t) {
@@ -278,308 +238,600 @@ __device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmA
     const int rem = t - c.b * per;
     c.mt = rem / g.n_tiles;
     c.nt = rem - c.mt * g.n_tiles;
+    c.n0 = c.nt * g.BN;
+    c.bn = min(g.BN, g.Ncols - c.n0);
     c.kb_end = g.k_blocks;
-    if (g.tri) c.kb_end = min(g.k_blocks, ((c.nt + 1) * g.BN + BK - 1) / BK);
-    const MatWork& w = batch.w[c.b];
-    if (EPI == EPI_STORE) c.active = g.st.active(w);
-    else c.active = !(*w.status & ST_FAILED);
+    if (g.tri) c.kb_end = min(g.k_blocks, (c.n0 + c.bn + BK - 1) / BK);
+    const int st = *batch.w[c.b].status;
+    c.active = !(st & ST_FAILED);
+    if (EPI != EPI_K5 && g.out.only_if_shifted && !(st & g.out.shift_bit)) c.active = false;
+    if (g.lower_only && c.n0 > c.mt * BM + BM - 1) c.active = false;
     return c;
 }
 
-template <int AMODE, int EPI>
-__global__ void __launch_bounds__(AMODE == A_PACKED ? THREADS_PACKED : THREADS_BUF, 1)
-umma_gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArgs g) {
+// N_IMG_MN: the pieces of depth block kb are its ks-deep slices that start below Kdim.
+__device__ __forceinline__ int mn_pieces(const GemmArgs& g, int kb) {
+    const int left = g.Kdim - kb * BK;
+    return (min(left, BK) + g.ks - 1) / g.ks;
+}
+// N_IMG_K: the pieces of depth block kb are 128-row chunks of the tile's N range; with a lower
+// triangular N-side a chunk is skipped once the depth block lies beyond its last row.
+__device__ __forceinline__ bool k_piece_active(const GemmArgs& g, const TileCoord& c, int kb, int chunk) {
+    return !g.tri || kb * BK <= c.n0 + min(c.bn, (chunk + 1) * 128) - 1;
+}
+
+// ------------------------------------------------------------------------------------------
+// The GEMM kernel.  D (128 x bn, fp32 in tensor memory) = A (128 x K) * N^T (bn x K).
+//   warp 0        producer: bulk copies of image tiles into the A ring and the N ring
+//   warp 1        MMA issuer, owns the tensor-memory allocation
+//   next 4 or 8   epilogue warps (tensor memory -> registers -> global)
+//   last 16       transform warps (A_BUF_* only): form B = M + G, split, write the A tile
+// AMODE  where the A tile comes from and how it lies in shared memory
+//          A_IMG_K / A_IMG_MN   image tile, K-major / MN-major
+//          A_BUF_ROW            rows of B = M + G      (K-major;  Y = B Q_prev, Alg. 1 line 2)
+//          A_BUF_COL            columns of B = M + G   (MN-major; R = B^T P,    Alg. 1 line 3)
+// NMODE  N_IMG_K   pieces = 128-row chunks of the N range, 64 deep (image K-major)
+//        N_IMG_MN  pieces = ks-deep slices of the whole N range (image MN-major)
+// EPI    EPI_STORE  fp32 copy and/or split image (+ column-square partials) of D
+//        EPI_K5     M <- a (M+G) - b D1,  X <- c X - d D2     (Alg. 1 lines 5-7), D1 = P R^T, D2 = P Q^T
+// XG     bit 0: G is bf16, bit 1: X is bf16
+// ------------------------------------------------------------------------------------------
+template <int XG>
+struct K5Pre {      // M, G, X of one 32 x 32 slab: 8 steps of (4 rows x 32 columns) per warp
+    float4 m[8];
+    uint32_t g[8][(XG & 1) ? 2 : 4];
+    uint32_t x[8][(XG & 2) ? 2 : 4];
+};
+
+template <int AMODE, int NMODE, int EPI, int XG>
+__global__ void __launch_bounds__(gemm_threads(AMODE, EPI), 1)
+gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArgs g) {
+    constexpr int NE = epi_warps(EPI);
+    constexpr bool A_BUF = a_is_buf(AMODE);
+    constexpr bool A_MN = (AMODE == A_IMG_MN || AMODE == A_BUF_COL);
+    constexpr bool G_BF16 = (XG & 1) != 0;
+    constexpr bool X_BF16 = (XG & 2) != 0;
+
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);
-    const int BN = g.BN;
-    const uint32_t b_term_bytes = (uint32_t)BN * 128u;
-    const uint32_t nb_ops = (EPI == EPI_K5) ? 2u : 1u;
-    const uint32_t stage_bytes = 2u * TILE_BYTES + 2u * b_term_bytes * nb_ops;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * stage_bytes);
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES;
-    const uint32_t tfull0 = empty0 + 8 * STAGES, tempty0 = tfull0 + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    unsigned char* a_ring = smem;
+    unsigned char* n_ring = smem + A_SLOTS * A_SLOT_BYTES;
+    unsigned char* staging = n_ring + (size_t)g.n_slots * g.n_piece_bytes;
+    unsigned char* tail = staging + (EPI == EPI_K5 ? NE * STAGING_BYTES_PER_WARP : 0);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
+    const uint32_t a_full0 = smem_u32(bars), a_empty0 = a_full0 + 8 * A_SLOTS;
+    const uint32_t n_full0 = a_empty0 + 8 * A_SLOTS, n_empty0 = n_full0 + 8 * MAX_N_SLOTS;
+    const uint32_t tfull0 = n_empty0 + 8 * MAX_N_SLOTS, tempty0 = tfull0 + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * A_SLOTS + 2 * MAX_N_SLOTS + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const uint32_t acc_cols = (EPI == EPI_K5) ? 2u * BN : (uint32_t)BN;
-    uint32_t alloc_cols = 32;
-    while (alloc_cols < 2 * acc_cols) alloc_cols *= 2;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full0 + 8 * s, AMODE == A_PACKED ? 1 : 1 + NUM_XF_WARPS);
-            mbar_init(empty0 + 8 * s, 1);
+        for (int s = 0; s < A_SLOTS; ++s) {
+            mbar_init(a_full0 + 8 * s, A_BUF ? NUM_XF_WARPS : 1);
+            mbar_init(a_empty0 + 8 * s, 1);
+        }
+        for (int s = 0; s < MAX_N_SLOTS; ++s) {
+            mbar_init(n_full0 + 8 * s, 1);
+            mbar_init(n_empty0 + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull0 + 8 * a, 1);
-            mbar_init(tempty0 + 8 * a, NUM_EPI_WARPS);
+            mbar_init(tempty0 + 8 * a, NE);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), alloc_cols);
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)g.tmem_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const uint32_t acc_stride = (uint32_t)(g.tmem_cols / g.acc_bufs);
 
     const int a_terms = (g.passes == 3 || (EPI == EPI_K5 && g.passes2 == 3)) ? 2 : 1;
-    const int b_terms = g.passes == 3 ? 2 : 1;
-    const int b2_terms = g.passes2 == 3 ? 2 : 1;
+    const int n1_terms = g.passes == 3 ? 2 : 1;
+    const int n2_terms = g.passes2 == 3 ? 2 : 1;
+    // N_IMG_MN piece geometry: [term][64-column group][ks rows of 128 bytes]
+    const uint32_t group_stride = (uint32_t)g.ks * 128u;
+    const uint32_t mn_term_stride = (uint32_t)((g.BN + 63) / 64) * group_stride;
 
     if (warp == 0) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            int stage = 0; uint32_t phase = 0;
+            int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                 const TileCoord c = decode_tile<EPI>(batch, g, t);
                 if (!c.active) continue;
                 const unsigned char* scr = reinterpret_cast<const unsigned char*>(batch.w[c.b].scratch);
-                const int n0 = c.nt * BN;
-                const int b_rt = n0 / 128;
-                const uint32_t b_row_off = (uint32_t)(n0 % 128) * 128u;
-                for (int kb = 0; kb < c.kb_end; ++kb) {
-                    if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                    unsigned char* sbase = smem + stage * stage_bytes;
-                    const uint32_t fb = full0 + 8 * stage;
-                    uint32_t bytes = b_terms * b_term_bytes;
-                    if (AMODE == A_PACKED) bytes += a_terms * TILE_BYTES;
-                    if (EPI == EPI_K5) bytes += b2_terms * b_term_bytes;
-                    mbar_arrive_expect_tx(fb, bytes);
-                    if (AMODE == A_PACKED) {
-                        for (int term = 0; term < a_terms; ++term) {
-                            const unsigned char* src = scr + g.a.off +
-                                ((int64_t)(kb * g.a.terms + term) * g.a.row_tiles + c.mt) * TILE_BYTES;
-                            bulk_copy_g2s(smem_u32(sbase + term * TILE_BYTES), src, TILE_BYTES, fb);
+                for (int kb = 0; kb < c.kb_end && ok; ++kb) {
+                    if (!A_BUF) {
+                        if (!mbar_wait(a_empty0 + 8 * as, aph ^ 1, abort_flag)) { ok = false; break; }
+                        const uint32_t fb = a_full0 + 8 * as;
+                        const uint32_t dst = smem_u32(a_ring + as * A_SLOT_BYTES);
+                        if (AMODE == A_IMG_K) {
+                            mbar_arrive_expect_tx(fb, (uint32_t)a_terms * A_TERM_BYTES);
+                            for (int term = 0; term < a_terms; ++term)
+                                bulk_copy_g2s(dst + term * A_TERM_BYTES,
+                                              scr + img_row_offset(g.a, term, kb, (int64_t)c.mt * BM), A_TERM_BYTES, fb);
+                        } else {
+                            const int ng = min(2, g.a.panels - c.mt * 2);
+                            mbar_arrive_expect_tx(fb, (uint32_t)(a_terms * ng) * 8192u);
+                            for (int term = 0; term < a_terms; ++term)
+                                for (int gi = 0; gi < ng; ++gi)
+                                    bulk_copy_g2s(dst + term * A_TERM_BYTES + gi * 8192,
+                                                  scr + img_row_offset(g.a, term, c.mt * 2 + gi, (int64_t)kb * BK), 8192, fb);
+                        }
+                        if (++as == A_SLOTS) { as = 0; aph ^= 1; }
+                    }
+                    if (NMODE == N_IMG_MN) {
+                        const int pieces = mn_pieces(g, kb);
+                        const int np = (c.bn + 63) / 64, p0 = c.n0 / 64;
+                        for (int sub = 0; sub < pieces && ok; ++sub) {
+                            if (!mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag)) { ok = false; break; }
+                            const uint32_t fb = n_full0 + 8 * ns;
+                            const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                            mbar_arrive_expect_tx(fb, (uint32_t)(n1_terms * np) * group_stride);
+                            for (int term = 0; term < n1_terms; ++term)
+                                for (int i = 0; i < np; ++i)
+                                    bulk_copy_g2s(dst + term * mn_term_stride + i * group_stride,
+                                                  scr + img_row_offset(g.n1, term, p0 + i, (int64_t)kb * BK + sub * g.ks),
+                                                  group_stride, fb);
+                            if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
+                        }
+                    } else {
+                        const int chunks = (c.bn + 127) / 128;
+                        for (int ch = 0; ch < chunks && ok; ++ch) {
+                            if (!k_piece_active(g, c, kb, ch)) continue;
+                            if (!mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag)) { ok = false; break; }
+                            const uint32_t fb = n_full0 + 8 * ns;
+                            const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                            const int nt_all = n1_terms + (EPI == EPI_K5 ? n2_terms : 0);
+                            mbar_arrive_expect_tx(fb, (uint32_t)nt_all * A_TERM_BYTES);
+                            for (int term = 0; term < n1_terms; ++term)
+                                bulk_copy_g2s(dst + term * A_TERM_BYTES,
+                                              scr + img_row_offset(g.n1, term, kb, (int64_t)c.n0 + ch * 128), A_TERM_BYTES, fb);
+                            if (EPI == EPI_K5)
+                                for (int term = 0; term < n2_terms; ++term)
+                                    bulk_copy_g2s(dst + (n1_terms + term) * A_TERM_BYTES,
+                                                  scr + img_row_offset(g.n2, term, kb, (int64_t)c.n0 + ch * 128), A_TERM_BYTES, fb);
+                            if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
                         }
                     }
-                    for (int term = 0; term < b_terms; ++term) {
-                        const unsigned char* src = scr + g.b.off +
-                            ((int64_t)(kb * g.b.terms + term) * g.b.row_tiles + b_rt) * TILE_BYTES + b_row_off;
-                        bulk_copy_g2s(smem_u32(sbase + 2 * TILE_BYTES + term * b_term_bytes), src, b_term_bytes, fb);
-                    }
-                    if (EPI == EPI_K5) {
-                        for (int term = 0; term < b2_terms; ++term) {
-                            const unsigned char* src = scr + g.b2.off +
-                                ((int64_t)(kb * g.b2.terms + term) * g.b2.row_tiles + b_rt) * TILE_BYTES + b_row_off;
-                            bulk_copy_g2s(smem_u32(sbase + 2 * TILE_BYTES + (2 + term) * b_term_bytes), src,
-                                          b_term_bytes, fb);
-                        }
-                    }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        int stage = 0; uint32_t phase = 0;
+        int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
         int acc = 0; uint32_t acc_phase = 0;
         bool ok = true;
-        const uint32_t idesc = instr_desc((uint32_t)BN, AMODE == A_BUF_COL ? 1u : 0u);
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
             const TileCoord c = decode_tile<EPI>(batch, g, t);
             if (!c.active) continue;
             if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t d1 = tmem_base + acc * acc_cols;
-            const uint32_t d2 = d1 + BN;
-            for (int kb = 0; kb < c.kb_end; ++kb) {
-                if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
+            const uint32_t dacc = tmem_base + acc * acc_stride;
+            for (int kb = 0; kb < c.kb_end && ok; ++kb) {
+                if (!mbar_wait(a_full0 + 8 * as, aph, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t sa = smem_u32(smem + stage * stage_bytes);
-                    const uint32_t sb = sa + 2 * TILE_BYTES;
-#pragma unroll
-                    for (int j = 0; j < BK / 16; ++j) {
-                        uint64_t a0, a1;
-                        if (AMODE == A_BUF_COL) {
-                            // MN-major A: 64-column groups 8192 bytes apart, 8-deep groups 1024 bytes apart
-                            a0 = smem_desc(sa + j * 2048, 8192, 1024);
-                            a1 = smem_desc(sa + TILE_BYTES + j * 2048, 8192, 1024);
-                        } else {
-                            a0 = smem_desc(sa + j * 32, 16, 1024);
-                            a1 = smem_desc(sa + TILE_BYTES + j * 32, 16, 1024);
-                        }
-                        const uint64_t b0 = smem_desc(sb + j * 32, 16, 1024);
-                        const uint64_t b1 = smem_desc(sb + b_term_bytes + j * 32, 16, 1024);
-                        const uint32_t first = (kb > 0 || j > 0) ? 1u : 0u;
-                        umma_bf16(d1, a0, b0, idesc, first);
-                        if (g.passes == 3) {
-                            umma_bf16(d1, a0, b1, idesc, 1u);
-                            umma_bf16(d1, a1, b0, idesc, 1u);
-                        }
-                        if (EPI == EPI_K5) {
-                            const uint64_t c0 = smem_desc(sb + 2 * b_term_bytes + j * 32, 16, 1024);
-                            const uint64_t c1 = smem_desc(sb + 3 * b_term_bytes + j * 32, 16, 1024);
-                            umma_bf16(d2, a0, c0, idesc, first);
-                            if (g.passes2 == 3) {
-                                umma_bf16(d2, a0, c1, idesc, 1u);
-                                umma_bf16(d2, a1, c0, idesc, 1u);
+                const uint32_t sa = smem_u32(a_ring + as * A_SLOT_BYTES);
+                if (NMODE == N_IMG_MN) {
+                    const int pieces = mn_pieces(g, kb);
+                    for (int sub = 0; sub < pieces && ok; ++sub) {
+                        if (!mbar_wait(n_full0 + 8 * ns, nph, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        if (lane == 0) {
+                            const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                            const int k0 = kb * BK + sub * g.ks;
+                            const int nsl = (min(g.ks, g.Kdim - k0) + 15) / 16;
+                            for (int j = 0; j < nsl; ++j) {
+                                const int slice = sub * (g.ks / 16) + j;
+                                const uint64_t a0 = A_MN ? smem_desc(sa + slice * 2048, 8192, 1024)
+                                                         : smem_desc(sa + slice * 32, 16, 1024);
+                                const uint64_t a1 = A_MN ? smem_desc(sa + A_TERM_BYTES + slice * 2048, 8192, 1024)
+                                                         : smem_desc(sa + A_TERM_BYTES + slice * 32, 16, 1024);
+                                const uint32_t accum = (kb > 0 || sub > 0 || j > 0) ? 1u : 0u;
+                                for (int cc = 0; cc < c.bn; cc += 256) {
+                                    const uint32_t ncols = (uint32_t)min(256, c.bn - cc);
+                                    const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 1u);
+                                    const uint32_t nb = sn + (cc / 64) * group_stride + j * 2048;
+                                    const uint64_t b0 = smem_desc(nb, group_stride, 1024);
+                                    const uint64_t b1 = smem_desc(nb + mn_term_stride, group_stride, 1024);
+                                    umma_bf16(dacc + cc, a0, b0, idesc, accum);
+                                    if (g.passes == 3) {
+                                        umma_bf16(dacc + cc, a0, b1, idesc, 1u);
+                                        umma_bf16(dacc + cc, a1, b0, idesc, 1u);
+                                    }
+                                }
                             }
+                            umma_commit(n_empty0 + 8 * ns);
                         }
+                        __syncwarp();
+                        if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
                     }
-                    umma_commit(empty0 + 8 * stage);
+                } else {
+                    const int chunks = (c.bn + 127) / 128;
+                    const int nsl = min(4, (g.Kdim - kb * BK + 15) / 16);
+                    for (int ch = 0; ch < chunks && ok; ++ch) {
+                        if (!k_piece_active(g, c, kb, ch)) continue;
+                        if (!mbar_wait(n_full0 + 8 * ns, nph, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        if (lane == 0) {
+                            const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                            const uint32_t ncols = (uint32_t)min(128, c.bn - ch * 128);
+                            const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u);
+                            for (int j = 0; j < nsl; ++j) {
+                                const uint64_t a0 = A_MN ? smem_desc(sa + j * 2048, 8192, 1024)
+                                                         : smem_desc(sa + j * 32, 16, 1024);
+                                const uint64_t a1 = A_MN ? smem_desc(sa + A_TERM_BYTES + j * 2048, 8192, 1024)
+                                                         : smem_desc(sa + A_TERM_BYTES + j * 32, 16, 1024);
+                                const uint64_t b0 = smem_desc(sn + j * 32, 16, 1024);
+                                const uint64_t b1 = smem_desc(sn + A_TERM_BYTES + j * 32, 16, 1024);
+                                const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
+                                const uint32_t d1 = dacc + ch * 128;
+                                umma_bf16(d1, a0, b0, idesc, accum);
+                                if (g.passes == 3) {
+                                    umma_bf16(d1, a0, b1, idesc, 1u);
+                                    umma_bf16(d1, a1, b0, idesc, 1u);
+                                }
+                                if (EPI == EPI_K5) {
+                                    const uint32_t s2 = sn + n1_terms * A_TERM_BYTES;
+                                    const uint64_t c0 = smem_desc(s2 + j * 32, 16, 1024);
+                                    const uint64_t c1 = smem_desc(s2 + A_TERM_BYTES + j * 32, 16, 1024);
+                                    const uint32_t d2 = dacc + g.BN;
+                                    umma_bf16(d2, a0, c0, idesc, accum);
+                                    if (g.passes2 == 3) {
+                                        umma_bf16(d2, a0, c1, idesc, 1u);
+                                        umma_bf16(d2, a1, c0, idesc, 1u);
+                                    }
+                                }
+                            }
+                            umma_commit(n_empty0 + 8 * ns);
+                        }
+                        __syncwarp();
+                        if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
+                    }
                 }
+                if (!ok) break;
+                if (lane == 0) umma_commit(a_empty0 + 8 * as);
                 __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                if (++as == A_SLOTS) { as = 0; aph ^= 1; }
             }
             if (!ok) break;
             if (lane == 0) umma_commit(tfull0 + 8 * acc);
             __syncwarp();
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
         }
-    } else if (warp < 2 + NUM_EPI_WARPS) {
+    } else if (warp < 2 + NE) {
         // ---------------- epilogue ----------------
         int acc = 0; uint32_t acc_phase = 0;
         bool ok = true;
         const int quarter = warp % 4;                    // tensor-memory lanes 32*quarter .. +31
-        for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-            const TileCoord c = decode_tile<EPI>(batch, g, t);
-            if (!c.active) continue;
-            if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const MatWork& w = batch.w[c.b];
-            const uint32_t taddr = tmem_base + acc * acc_cols + ((uint32_t)(quarter * 32) << 16);
-            const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + lane;
-            const int n0 = c.nt * BN;
-            if (EPI == EPI_STORE) {
+        if (EPI == EPI_STORE) {
+            for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
+                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                if (!c.active) continue;
+                if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const MatWork& w = batch.w[c.b];
                 const int stw = *w.status;
-                float* C = pick(w, (g.st.shift_bit && (stw & g.st.shift_bit)) ? g.st.dst_if_shifted : g.st.dst);
-                for (int cc = 0; cc < BN; cc += 16) {
+                const Dest& d = (g.out.shift_bit && (stw & g.out.shift_bit)) ? g.out.shifted : g.out.normal;
+                const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16);
+                const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + lane;
+                float* C = d.has_f32 ? pick(w, d.f32) : nullptr;
+                unsigned char* scr = reinterpret_cast<unsigned char*>(w.scratch);
+                const bool to_img = d.img.off >= 0;
+                float* csq = d.colsq ? reinterpret_cast<float*>(w.scratch + g.colsq_off) +
+                                           (int64_t)(c.mt * 4 + quarter) * g.Ncols : nullptr;
+                const int bn64 = to_img ? (c.bn + 63) / 64 * 64 : c.bn;
+                for (int cc = 0; cc < bn64; cc += 16) {
                     uint32_t v[16];
-                    tmem_ld16(taddr + cc, v);
-                    tmem_ld_wait();
-                    if (gi < g.Mrows) {
+                    if (cc < c.bn) {
+                        tmem_ld16(taddr + cc, v);
+                        tmem_ld_wait();
+                    } else {
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int gj = n0 + cc + 4 * u;
-                            if (gj < g.Ncols)
-                                *reinterpret_cast<uint4*>(C + gi * g.st.ld + gj) =
-                                    make_uint4(v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
-                        }
+                        for (int i = 0; i < 16; ++i) v[i] = 0u;
                     }
-                }
-            } else {
-                for (int cc = 0; cc < BN; cc += 16) {
-                    uint32_t v1[16], v2[16];
-                    tmem_ld16(taddr + cc, v1);
-                    tmem_ld16(taddr + BN + cc, v2);
-                    tmem_ld_wait();
-                    if (gi < g.Mrows) {
+                    const int gj = c.n0 + cc;
+                    if (C && gi < g.Mrows && cc < c.bn) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            *reinterpret_cast<uint4*>(C + gi * g.out.ld + gj + 4 * u) =
+                                make_uint4(v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
+                    }
+                    if (to_img) {
+                        const int panel = gj / 64, ch0 = (gj % 64) / 8;
+                        unsigned char* r0 = scr + img_row_offset(d.img, 0, panel, gi);
+                        unsigned char* r1 = scr + img_row_offset(d.img, 1, panel, gi);
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const int gj = n0 + cc + 8 * h;
-                            if (gj < g.Ncols) {     // Ncols % 8 == 0
-                                const int64_t idx = gi * g.ld + gj;
-                                float mv[8], gv[8], xv[8];
-                                load8(w.M, idx, 0, mv);
-                                load8(w.G, idx, g.g_bf16, gv);
-                                load8(w.X, idx, g.x_bf16, xv);
-                                float mo[8], xo[8];
+                            float f[8];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const float bval = mv[e] + gv[e];
-                                    mo[e] = g.ef_a * bval - g.ef_b * __uint_as_float(v1[8 * h + e]);
-                                    xo[e] = g.wc * xv[e] - g.wd * __uint_as_float(v2[8 * h + e]);
-                                }
-                                float4* mp = reinterpret_cast<float4*>(w.M + idx);
-                                mp[0] = make_float4(mo[0], mo[1], mo[2], mo[3]);
-                                mp[1] = make_float4(mo[4], mo[5], mo[6], mo[7]);
-                                if (g.x_bf16) {
-                                    uint4 xp = make_uint4(pack_bf16x2(xo[0], xo[1]), pack_bf16x2(xo[2], xo[3]),
-                                                          pack_bf16x2(xo[4], xo[5]), pack_bf16x2(xo[6], xo[7]));
-                                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(w.X) + idx) = xp;
-                                } else {
-                                    float4* xp = reinterpret_cast<float4*>(reinterpret_cast<float*>(w.X) + idx);
-                                    xp[0] = make_float4(xo[0], xo[1], xo[2], xo[3]);
-                                    xp[1] = make_float4(xo[4], xo[5], xo[6], xo[7]);
+                            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * h + i]);
+                            uint4 t0, t1;
+                            split8(f, t0, t1);
+                            const int o = img_chunk_offset((int)(gi & 7), ch0 + h);
+                            *reinterpret_cast<uint4*>(r0 + o) = t0;
+                            *reinterpret_cast<uint4*>(r1 + o) = t1;
+                        }
+                    }
+                    if (csq && cc < c.bn) {
+                        // column sums of squares over the 32 rows of this warp: fold 16 values over
+                        // the lane bits 4..1, then add the two lanes that hold the same column
+                        float s[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { const float x = __uint_as_float(v[i]); s[i] = x * x; }
+#pragma unroll
+                        for (int half = 8, bit = 16; half >= 1; half >>= 1, bit >>= 1) {
+                            const bool up = (lane & bit) != 0;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (i < half) {
+                                    const float send = up ? s[i] : s[i + half];
+                                    const float keep = up ? s[i + half] : s[i];
+                                    s[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
                                 }
                             }
                         }
+                        s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
+                        const int col = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+                        if (!(lane & 1)) csq[gj + col] = s[0];
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        } else {
+            // Fused error feedback and weight update.  Warp (quarter, half) owns rows
+            // 32*quarter.. of the tile and columns 64*half.., in two slabs of 32 x 32.  The two
+            // accumulator slabs go through a swizzled staging block so that global accesses run
+            // along rows (8 lanes x 16 bytes per row); M, G, X of the next slab are fetched
+            // before the current one is finished.
+            constexpr bool PF = G_BF16 && X_BF16;
+            const int half = (warp - 2) / 4;
+            unsigned char* S1 = staging + (warp - 2) * STAGING_BYTES_PER_WARP;
+            unsigned char* S2 = S1 + 4096;
+            const int rl = lane / 8, cq = lane % 8;      // row within a step, 4-column group
+
+            auto next_tile = [&](int t) {
+                for (t += gridDim.x; t < g.total_tiles; t += gridDim.x)
+                    if (decode_tile<EPI>(batch, g, t).active) return t;
+                return g.total_tiles;
+            };
+            auto fetch = [&](K5Pre<XG>& p, int t, int slab) {
+                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                const MatWork& w = batch.w[c.b];
+                const int64_t gj = (int64_t)c.n0 + half * 64 + slab * 32 + cq * 4;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + it * 4 + rl;
+                    if (gi < g.Mrows && gj < g.Ncols) {
+                        const int64_t idx = gi * g.ld + gj;
+                        p.m[it] = *reinterpret_cast<const float4*>(w.M + idx);
+                        if constexpr (G_BF16) {
+                            const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(w.G) + idx);
+                            p.g[it][0] = u.x; p.g[it][1] = u.y;
+                        } else {
+                            const uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(w.G) + idx);
+                            p.g[it][0] = u.x; p.g[it][1] = u.y; p.g[it][2] = u.z; p.g[it][3] = u.w;
+                        }
+                        if constexpr (X_BF16) {
+                            const uint2 u = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(w.X) + idx);
+                            p.x[it][0] = u.x; p.x[it][1] = u.y;
+                        } else {
+                            const uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(w.X) + idx);
+                            p.x[it][0] = u.x; p.x[it][1] = u.y; p.x[it][2] = u.z; p.x[it][3] = u.w;
+                        }
+                    }
+                }
+            };
+
+            K5Pre<XG> pre, cur;
+            int t = blockIdx.x - (int)gridDim.x;
+            t = next_tile(t);
+            int slab = 0;
+            if (PF && t < g.total_tiles) fetch(pre, t, 0);
+            while (t < g.total_tiles && ok) {
+                int t2 = t, slab2 = slab + 1;
+                if (slab2 == 2) { slab2 = 0; t2 = next_tile(t); }
+                if constexpr (PF) {
+                    cur = pre;
+                    if (t2 < g.total_tiles) fetch(pre, t2, slab2);
+                } else {
+                    fetch(cur, t, slab);
+                }
+                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                const MatWork& w = batch.w[c.b];
+                if (slab == 0) {
+                    if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                }
+                const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16) +
+                                       (uint32_t)(half * 64 + slab * 32);
+                {
+                    uint32_t v1[32], v2[32];
+                    tmem_ld16(taddr, *reinterpret_cast<uint32_t(*)[16]>(&v1[0]));
+                    tmem_ld16(taddr + 16, *reinterpret_cast<uint32_t(*)[16]>(&v1[16]));
+                    tmem_ld16(taddr + g.BN, *reinterpret_cast<uint32_t(*)[16]>(&v2[0]));
+                    tmem_ld16(taddr + g.BN + 16, *reinterpret_cast<uint32_t(*)[16]>(&v2[16]));
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        const int o = lane * 128 + img_chunk_offset(lane, ch);
+                        *reinterpret_cast<uint4*>(S1 + o) = make_uint4(v1[4 * ch], v1[4 * ch + 1], v1[4 * ch + 2], v1[4 * ch + 3]);
+                        *reinterpret_cast<uint4*>(S2 + o) = make_uint4(v2[4 * ch], v2[4 * ch + 1], v2[4 * ch + 2], v2[4 * ch + 3]);
+                    }
+                }
+                __syncwarp();
+                const int64_t gj = (int64_t)c.n0 + half * 64 + slab * 32 + cq * 4;
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int r = it * 4 + rl;
+                    const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + r;
+                    const int o = r * 128 + img_chunk_offset(r, cq);
+                    const float4 d1 = *reinterpret_cast<const float4*>(S1 + o);
+                    const float4 d2 = *reinterpret_cast<const float4*>(S2 + o);
+                    if (gi < g.Mrows && gj < g.Ncols) {
+                        const int64_t idx = gi * g.ld + gj;
+                        float gv[4], xv[4];
+                        if constexpr (G_BF16) {
+                            gv[0] = bf16lo_to_f32(cur.g[it][0]); gv[1] = bf16hi_to_f32(cur.g[it][0]);
+                            gv[2] = bf16lo_to_f32(cur.g[it][1]); gv[3] = bf16hi_to_f32(cur.g[it][1]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) gv[e] = __uint_as_float(cur.g[it][e]);
+                        }
+                        if constexpr (X_BF16) {
+                            xv[0] = bf16lo_to_f32(cur.x[it][0]); xv[1] = bf16hi_to_f32(cur.x[it][0]);
+                            xv[2] = bf16lo_to_f32(cur.x[it][1]); xv[3] = bf16hi_to_f32(cur.x[it][1]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) xv[e] = __uint_as_float(cur.x[it][e]);
+                        }
+                        const float mv[4] = {cur.m[it].x, cur.m[it].y, cur.m[it].z, cur.m[it].w};
+                        const float a1[4] = {d1.x, d1.y, d1.z, d1.w};
+                        const float a2[4] = {d2.x, d2.y, d2.z, d2.w};
+                        float mo[4], xo[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float bval = mv[e] + gv[e];
+                            mo[e] = g.ef_a * bval - g.ef_b * a1[e];
+                            xo[e] = g.wc * xv[e] - g.wd * a2[e];
+                        }
+                        *reinterpret_cast<float4*>(w.M + idx) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+                        if constexpr (X_BF16) {
+                            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(w.X) + idx) =
+                                make_uint2(pack_bf16x2(xo[0], xo[1]), pack_bf16x2(xo[2], xo[3]));
+                        } else {
+                            *reinterpret_cast<float4*>(reinterpret_cast<float*>(w.X) + idx) =
+                                make_float4(xo[0], xo[1], xo[2], xo[3]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (slab == 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                    if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
+                }
+                t = t2; slab = slab2;
+            }
         }
-    } else if (AMODE != A_PACKED) {
-        // ---------------- transform warps: A image of B = M + G ----------------
-        const int xt = threadIdx.x - 32 * (2 + NUM_EPI_WARPS);     // 0 .. 255
-        int stage = 0; uint32_t phase = 0;
+    } else if (A_BUF) {
+        // ---------------- transform warps: A tile of B = M + G (Alg. 1 line 1) ----------------
+        // 512 threads, two 8-element chunks each per 128 x 64 tile; the loads of the next two
+        // tiles are in flight while the current one is split and stored.
+        const int xt = threadIdx.x - 32 * (2 + NE);     // 0 .. 511
+        int as = 0; uint32_t aph = 0;
         bool ok = true;
+        struct Raw { float4 m[2][2]; uint32_t gq[2][G_BF16 ? 4 : 8]; };
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
             const TileCoord c = decode_tile<EPI>(batch, g, t);
             if (!c.active) continue;
             const MatWork& w = batch.w[c.b];
             const int64_t ld = g.ld;
-            // chunk coordinates of this thread (4 chunks per stage)
-            int64_t src_idx[4]; bool row_ok[4]; int kofs[4]; uint32_t dst_off[4];
+            int64_t src_idx[2]; bool row_ok[2]; int kofs[2]; uint32_t dst_off[2];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int q = xt + 256 * e;
+            for (int e = 0; e < 2; ++e) {
+                const int q = xt + 512 * e;
                 if (AMODE == A_BUF_ROW) {
-                    // operand row = B row, depth = B column: chunk (rho, c) = B[i0+rho][k0+8c .. +7]
+                    // operand row = B row, depth = B column: chunk (rho, ch) = B[i0+rho][k0+8ch .. +7]
                     const int rho = q / 8, ch = q % 8;
                     const int64_t gr = (int64_t)c.mt * BM + rho;
                     row_ok[e] = gr < g.Mrows;
                     src_idx[e] = gr * ld + ch * 8;           // + k0
                     kofs[e] = ch * 8;
-                    dst_off[e] = rho * 128 + ((ch ^ (rho & 7)) << 4);
+                    dst_off[e] = rho * 128 + img_chunk_offset(rho, ch);
                 } else {
-                    // operand row = B column, depth = B row (MN-major image):
+                    // operand row = B column, depth = B row (MN-major tile):
                     // chunk (k, cj) = B[k0+k][j0+8cj .. +7]
                     const int k = q / 16, cj = q % 16;
                     const int64_t gc = (int64_t)c.mt * BM + cj * 8;
-                    row_ok[e] = gc < g.Mrows;                // Mrows = number of B columns (n), n % 8 == 0
+                    row_ok[e] = gc < g.Mrows;                // Mrows = number of B columns, a multiple of 8
                     src_idx[e] = (int64_t)k * ld + gc;       // + k0 * ld
                     kofs[e] = k;
-                    dst_off[e] = (cj / 8) * 8192 + (k / 8) * 1024 + (k % 8) * 128 + (((cj % 8) ^ (k % 8)) << 4);
+                    dst_off[e] = (cj / 8) * 8192 + k * 128 + img_chunk_offset(k, cj % 8);
                 }
             }
-            float mv[4][8], gv[4][8];
-            auto fetch = [&](int kb) {
+            auto fetch = [&](Raw& r, int kb) {
+                const int64_t k0 = (int64_t)kb * BK;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int64_t k0 = (int64_t)kb * BK;
-                    bool okk = row_ok[e] && (k0 + kofs[e] < g.Kdim);
+                for (int e = 0; e < 2; ++e) {
+                    const bool okk = row_ok[e] && (k0 + kofs[e] < g.Kdim);
                     if (okk) {
                         const int64_t idx = src_idx[e] + (AMODE == A_BUF_ROW ? k0 : k0 * ld);
-                        load8(w.M, idx, 0, mv[e]);
-                        load8(w.G, idx, g.g_bf16, gv[e]);
+                        const float4* mp = reinterpret_cast<const float4*>(w.M + idx);
+                        r.m[e][0] = mp[0]; r.m[e][1] = mp[1];
+                        if constexpr (G_BF16) {
+                            const uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(w.G) + idx);
+                            r.gq[e][0] = u.x; r.gq[e][1] = u.y; r.gq[e][2] = u.z; r.gq[e][3] = u.w;
+                        } else {
+                            const uint4* gp = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(w.G) + idx);
+                            const uint4 u0 = gp[0], u1 = gp[1];
+                            r.gq[e][0] = u0.x; r.gq[e][1] = u0.y; r.gq[e][2] = u0.z; r.gq[e][3] = u0.w;
+                            r.gq[e][4] = u1.x; r.gq[e][5] = u1.y; r.gq[e][6] = u1.z; r.gq[e][7] = u1.w;
+                        }
                     } else {
+                        r.m[e][0] = r.m[e][1] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) { mv[e][i] = 0.f; gv[e][i] = 0.f; }
+                        for (int i = 0; i < (G_BF16 ? 4 : 8); ++i) r.gq[e][i] = 0u;
                     }
                 }
             };
-            fetch(0);
-            for (int kb = 0; kb < c.kb_end; ++kb) {
-                uint4 t0[4], t1[4];
+            // split the tile held in r into the two bf16 terms
+            auto split_raw = [&](const Raw& r, uint4 (&t0)[2], uint4 (&t1)[2]) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v[8];
+                for (int e = 0; e < 2; ++e) {
+                    float gv[8];
+                    if constexpr (G_BF16) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) v[i] = mv[e][i] + gv[e][i];
+                        for (int i = 0; i < 4; ++i) { gv[2 * i] = bf16lo_to_f32(r.gq[e][i]); gv[2 * i + 1] = bf16hi_to_f32(r.gq[e][i]); }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) gv[i] = __uint_as_float(r.gq[e][i]);
+                    }
+                    const float v[8] = {r.m[e][0].x + gv[0], r.m[e][0].y + gv[1], r.m[e][0].z + gv[2], r.m[e][0].w + gv[3],
+                                        r.m[e][1].x + gv[4], r.m[e][1].y + gv[5], r.m[e][1].z + gv[6], r.m[e][1].w + gv[7]};
                     split8(v, t0[e], t1[e]);
                 }
-                if (kb + 1 < c.kb_end) fetch(kb + 1);
-                if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                unsigned char* sa = smem + stage * stage_bytes;
+            };
+            // wait for the slot, store the tile, signal the MMA issuer
+            auto store = [&](const uint4 (&t0)[2], const uint4 (&t1)[2]) -> bool {
+                if (!mbar_wait(a_empty0 + 8 * as, aph ^ 1, abort_flag)) return false;
+                unsigned char* sa = a_ring + as * A_SLOT_BYTES;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
+                for (int e = 0; e < 2; ++e) {
                     *reinterpret_cast<uint4*>(sa + dst_off[e]) = t0[e];
-                    *reinterpret_cast<uint4*>(sa + TILE_BYTES + dst_off[e]) = t1[e];
+                    *reinterpret_cast<uint4*>(sa + A_TERM_BYTES + dst_off[e]) = t1[e];
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(full0 + 8 * stage);
-                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                if (lane == 0) mbar_arrive(a_full0 + 8 * as);
+                if (++as == A_SLOTS) { as = 0; aph ^= 1; }
+                return true;
+            };
+            Raw r0, r1;
+            fetch(r0, 0);
+            if (c.kb_end > 1) fetch(r1, 1);
+            for (int kb = 0; kb < c.kb_end && ok; kb += 2) {
+                uint4 t0[2], t1[2];
+                split_raw(r0, t0, t1);
+                if (kb + 2 < c.kb_end) fetch(r0, kb + 2);
+                if (!store(t0, t1)) { ok = false; break; }
+                if (kb + 1 < c.kb_end) {
+                    split_raw(r1, t0, t1);
+                    if (kb + 3 < c.kb_end) fetch(r1, kb + 3);
+                    if (!store(t0, t1)) { ok = false; break; }
+                }
             }
         }
     }
@@ -591,20 +843,7 @@ umma_gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ Ge
     if (*abort_flag && threadIdx.x == 0) {
         for (int b = 0; b < batch.count; ++b) atomicOr(batch.w[b].status, ST_WAIT);
     }
-    if (warp == 1) tmem_dealloc(tmem_base, alloc_cols);
-}
-
-// smem bytes a launch asks for: the stages, barriers, alignment slack, and enough to keep the number
-// of resident CTAs per SM times their tensor-memory columns within the 512 columns of an SM.
-inline size_t gemm_smem_bytes(int BN, bool k5) {
-    const size_t stage = 2 * (size_t)TILE_BYTES + 2 * (size_t)BN * 128 * (k5 ? 2 : 1);
-    size_t need = STAGES * stage + 256 + 1024;
-    const size_t acc = (size_t)(k5 ? 2 * BN : BN);
-    size_t cols = 32;
-    while (cols < 2 * acc) cols *= 2;
-    const size_t max_resident = 512 / cols;
-    const size_t min_smem = (227 * 1024) / (max_resident + 1) + 1024;
-    return std::max(need, max_resident >= 8 ? need : min_smem);
+    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)g.tmem_cols);
 }
 
 }  // namespace tc
@@ -612,52 +851,51 @@ inline size_t gemm_smem_bytes(int BN, bool k5) {
 // ------------------------------------------------------------------------------------------
 // Host side of the engine
 // ------------------------------------------------------------------------------------------
-struct TensorScratch {
-    int64_t q_t, src_t, src_n, linv, p_t, p_n, r_n, q_n;   // byte offsets of the packed operands
-    int64_t colsq;                                          // fp32 [kblocks][r] column sums of squares
+struct TensorScratch {      // where the images of one matrix live inside its scratch area
+    ImgRef linv;            // L^{-1} of the current Cholesky            (r x r)
+    ImgRef qprev;           // Q_prev                                    (n x r)
+    ImgRef w0, w1;          // Y = B Q_prev and the QR intermediates     (max(m,n) x r)
+    ImgRef p, r, q;         // P (m x r), R (n x r), Q (n x r)
+    int64_t colsq;          // fp32 [4 * ceil(max(m,n)/128)][r] column-square partials
 };
 
 inline bool tensor_engine_supports(int64_t m, int64_t n, int32_t r) {
     return r % 16 == 0 && n % 8 == 0 && m >= 1;
 }
 
-inline int64_t pack_bytes(int64_t rows, int64_t depth, int terms) {
-    return ((rows + 127) / 128) * ((depth + 63) / 64) * terms * (int64_t)tc::TILE_BYTES;
+inline ImgRef make_img(int64_t off, int64_t rows, int64_t cols) {
+    ImgRef im;
+    im.off = off;
+    im.rows_pad = (int32_t)((rows + 127) / 128 * 128);
+    im.panels = (int32_t)((cols + 63) / 64);
+    return im;
 }
+inline int64_t img_bytes(int64_t rows, int64_t cols) {
+    return 2 * ((cols + 63) / 64) * ((rows + 127) / 128 * 128) * 128;
+}
+inline ImgRef no_img() { ImgRef im; im.off = -1; im.rows_pad = 0; im.panels = 0; return im; }
 
+// The offsets of linv and colsq depend on r only, so that one Cholesky launch can serve
+// matrices of different shapes.
 inline size_t tensor_scratch_layout(int64_t m, int64_t n, int32_t r, size_t off, TensorScratch* ts) {
     const int64_t kmax = std::max(m, n);
-    auto take = [&](int64_t bytes) { int64_t o = (int64_t)off; off += (size_t)((bytes + 1023) / 1024 * 1024); return o; };
     off = (off + 1023) / 1024 * 1024;
-    ts->q_t = take(pack_bytes(r, n, 2));
-    ts->src_t = take(pack_bytes(r, kmax, 2));
-    ts->src_n = take(pack_bytes(kmax, r, 2));
-    ts->linv = take(pack_bytes(r, r, 2));
-    ts->p_t = take(pack_bytes(r, m, 2));
-    ts->p_n = take(pack_bytes(m, r, 2));
-    ts->r_n = take(pack_bytes(n, r, 2));
-    ts->q_n = take(pack_bytes(n, r, 2));
-    ts->colsq = take(((kmax + 63) / 64) * (int64_t)r * 4);
+    auto take = [&](int64_t bytes) { int64_t o = (int64_t)off; off += (size_t)((bytes + 1023) / 1024 * 1024); return o; };
+    ts->linv = make_img(take(img_bytes(r, r)), r, r);
+    ts->colsq = take(4 * ((kmax + 127) / 128) * (int64_t)r * 4);
+    ts->qprev = make_img(take(img_bytes(n, r)), n, r);
+    ts->w0 = make_img(take(img_bytes(kmax, r)), kmax, r);
+    ts->w1 = make_img(take(img_bytes(kmax, r)), kmax, r);
+    ts->p = make_img(take(img_bytes(m, r)), m, r);
+    ts->r = make_img(take(img_bytes(n, r)), n, r);
+    ts->q = make_img(take(img_bytes(n, r)), n, r);
     return off;
 }
-
-inline int tensor_bn(int64_t ncols) {
-    int bn = 16;
-    while (bn < 256 && bn < ncols) bn *= 2;
-    return bn;
-}
-
-inline cudaError_t tensor_engine_set_attributes() {
-    const int max_smem = 227 * 1024;
-    cudaError_t e;
-#define OD_SET(k) \
-    if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
-    OD_SET((tc::umma_gemm_kernel<tc::A_PACKED, tc::EPI_STORE>))
-    OD_SET((tc::umma_gemm_kernel<tc::A_PACKED, tc::EPI_K5>))
-    OD_SET((tc::umma_gemm_kernel<tc::A_BUF_ROW, tc::EPI_STORE>))
-    OD_SET((tc::umma_gemm_kernel<tc::A_BUF_COL, tc::EPI_STORE>))
-#undef OD_SET
-    return cudaSuccess;
+// the work images are sized for max(m, n) rows; a product over `rows` rows sees this view
+inline ImgRef img_view(const ImgRef& im, int64_t rows) {
+    ImgRef v = im;
+    v.rows_pad = (int32_t)((rows + 127) / 128 * 128);
+    return v;
 }
 
 inline int sm_count() {
@@ -671,113 +909,141 @@ inline int sm_count() {
     return n;
 }
 
-inline tc::PackRef make_pack(int64_t off, int64_t rows, int64_t depth, int terms) {
-    tc::PackRef p;
-    p.off = off;
-    p.row_tiles = (int32_t)((rows + 127) / 128);
-    p.terms = terms;
-    p.kblocks = (int32_t)((depth + 63) / 64);
-    p.pad = 0;
-    return p;
+template <int AMODE, int NMODE, int EPI, int XG>
+inline cudaError_t set_gemm_attr() {
+    return cudaFuncSetAttribute(tc::gemm_kernel<AMODE, NMODE, EPI, XG>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
 }
 
-// pack S (rows_s x cols_s) either as (operand rows = S rows) or transposed
-inline void launch_pack(const Batch& b, Sel src, int64_t rows_s, int64_t cols_s, int trans, tc::PackRef dst,
-                        int shift_bit_only, cudaStream_t st, int64_t colsq_off = -1) {
+inline cudaError_t tensor_engine_set_attributes() {
+    cudaError_t e;
+#define OD_SET(...) if ((e = set_gemm_attr<__VA_ARGS__>()) != cudaSuccess) return e;
+    OD_SET(tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 0)
+    OD_SET(tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 1)
+    OD_SET(tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 0)
+    OD_SET(tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 1)
+    OD_SET(tc::A_IMG_MN, tc::N_IMG_MN, tc::EPI_STORE, 0)
+    OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_STORE, 0)
+    OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 0)
+    OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 1)
+    OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 2)
+    OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 3)
+#undef OD_SET
+    return cudaSuccess;
+}
+
+inline void launch_pack(const Batch& b, Sel src, int64_t rows, int64_t cols, ImgRef dst, cudaStream_t st) {
     tc::PackArgs a{};
-    a.colsq_off = colsq_off; a.colsq_ld = (int32_t)cols_s;
-    a.src = src; a.rows_s = (int32_t)rows_s; a.cols_s = (int32_t)cols_s; a.trans = trans;
-    a.only_if_shifted = shift_bit_only ? 1 : 0; a.shift_bit = shift_bit_only; a.dst = dst;
-    dim3 grid((unsigned)dst.kblocks, (unsigned)dst.row_tiles, (unsigned)b.count);
+    a.src = src; a.rows = (int32_t)rows; a.cols = (int32_t)cols; a.dst = dst;
+    dim3 grid((unsigned)dst.panels, (unsigned)(dst.rows_pad / 128), (unsigned)b.count);
     prof::Scope scope(prof::S_PACK, st);
     tc::pack_kernel<<<grid, 256, 0, st>>>(b, a);
 }
 
-template <int AMODE, int EPI>
+// Fills in the tiling, ring and tensor-memory fields and launches.
+template <int AMODE, int NMODE, int EPI, int XG>
 inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t st) {
     g.m_tiles = (g.Mrows + tc::BM - 1) / tc::BM;
     g.n_tiles = (g.Ncols + g.BN - 1) / g.BN;
     g.k_blocks = (g.Kdim + tc::BK - 1) / tc::BK;
     g.total_tiles = b.count * g.m_tiles * g.n_tiles;
-    const size_t smem = tc::gemm_smem_bytes(g.BN, EPI == tc::EPI_K5);
-    const int per_sm = std::max<int>(1, (int)((227 * 1024) / smem));
-    const int grid = std::min(g.total_tiles, sm_count() * per_sm);
-    const int threads = AMODE == tc::A_PACKED ? tc::THREADS_PACKED : tc::THREADS_BUF;
+    const int n1_terms = g.passes == 3 ? 2 : 1, n2_terms = g.passes2 == 3 ? 2 : 1;
+    const int bn64 = (g.BN + 63) / 64 * 64;
+    if (NMODE == tc::N_IMG_MN) {
+        g.ks = bn64 <= 128 ? 64 : (bn64 <= 256 ? 32 : 16);
+        g.n_piece_bytes = n1_terms * (bn64 / 64) * g.ks * 128;
+    } else {
+        g.ks = 64;
+        g.n_piece_bytes = (n1_terms + (EPI == tc::EPI_K5 ? n2_terms : 0)) * tc::A_TERM_BYTES;
+    }
+    const int accw = (EPI == tc::EPI_K5) ? 2 * g.BN : g.BN;
+    g.acc_bufs = (2 * accw <= 512) ? 2 : 1;
+    int cols = 32;
+    while (cols < g.acc_bufs * accw) cols *= 2;
+    g.tmem_cols = cols;
+    const size_t fixed = (size_t)tc::A_SLOTS * tc::A_SLOT_BYTES +
+                         (EPI == tc::EPI_K5 ? tc::epi_warps(EPI) * tc::STAGING_BYTES_PER_WARP : 0) + 256 + 1024;
+    g.n_slots = (int)std::min<size_t>(tc::MAX_N_SLOTS, (tc::SMEM_LIMIT - fixed) / (size_t)g.n_piece_bytes);
+    // more than half of an SM's shared memory: one CTA per SM, whatever its tensor-memory share
+    const size_t smem = std::max<size_t>(fixed + (size_t)g.n_slots * g.n_piece_bytes, 120 * 1024);
+    const int grid = std::min(g.total_tiles, sm_count());
     prof::Scope scope(stage, st);
-    tc::umma_gemm_kernel<AMODE, EPI><<<grid, threads, smem, st>>>(b, g);
+    tc::gemm_kernel<AMODE, NMODE, EPI, XG><<<grid, tc::gemm_threads(AMODE, EPI), smem, st>>>(b, g);
 }
 
-// Y = (M + G) Q_prev  -> P slot                                   (Alg. 1 lines 1-2)
+inline tc::Dest dest_none() {
+    tc::Dest d{};
+    d.f32 = Sel{W_P, 0, 0}; d.img = no_img(); d.has_f32 = 0; d.colsq = 0;
+    return d;
+}
+
+// Y = (M + G) Q_prev  -> image w0 (+ column squares)              (Alg. 1 lines 1-2)
 inline void tensor_k1(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
                       cudaStream_t st) {
-    const int terms = passes == 3 ? 2 : 1;
-    tc::PackRef qt = make_pack(ts.q_t, r, n, terms);
-    launch_pack(b, Sel{W_Q, 0, 0}, n, r, 1, qt, 0, st);
+    launch_pack(b, Sel{W_Q, 0, 0}, n, r, ts.qprev, st);
     tc::GemmArgs g{};
-    g.Mrows = (int32_t)m; g.Ncols = r; g.Kdim = (int32_t)n; g.BN = tensor_bn(r);
-    g.passes = passes; g.passes2 = 1; g.g_bf16 = g_bf16; g.ld = n; g.b = qt;
-    g.st = EpStore{Sel{W_P, 0, 0}, Sel{W_P, 0, 0}, 0, 0, r, 0};
-    launch_gemm<tc::A_BUF_ROW, tc::EPI_STORE>(b, g, prof::S_K1, st);
+    g.Mrows = (int32_t)m; g.Ncols = r; g.Kdim = (int32_t)n; g.BN = std::min(r, 512);
+    g.passes = passes; g.passes2 = 1; g.ld = n; g.n1 = ts.qprev; g.a = no_img(); g.n2 = no_img();
+    g.colsq_off = ts.colsq;
+    g.out.normal = dest_none(); g.out.normal.img = img_view(ts.w0, m); g.out.normal.colsq = 1;
+    g.out.shifted = g.out.normal; g.out.ld = r;
+    if (g_bf16) launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 1>(b, g, prof::S_K1, st);
+    else launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K1, st);
 }
 
-// R = (M + G)^T P  -> R slot                                      (Alg. 1 line 3)
+// R = (M + G)^T P  -> fp32 R slot, image r (+ column squares)     (Alg. 1 line 3)
 inline void tensor_k3(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
                       cudaStream_t st) {
-    const int terms = passes == 3 ? 2 : 1;
-    tc::PackRef pt = make_pack(ts.p_t, r, m, terms);
-    launch_pack(b, Sel{W_P, 0, 0}, m, r, 1, pt, 0, st);
     tc::GemmArgs g{};
-    g.Mrows = (int32_t)n; g.Ncols = r; g.Kdim = (int32_t)m; g.BN = tensor_bn(r);
-    g.passes = passes; g.passes2 = 1; g.g_bf16 = g_bf16; g.ld = n; g.b = pt;
-    g.st = EpStore{Sel{W_R, 0, 0}, Sel{W_R, 0, 0}, 0, 0, r, 0};
-    launch_gemm<tc::A_BUF_COL, tc::EPI_STORE>(b, g, prof::S_K3, st);
+    g.Mrows = (int32_t)n; g.Ncols = r; g.Kdim = (int32_t)m; g.BN = std::min(r, 512);
+    g.passes = passes; g.passes2 = 1; g.ld = n; g.n1 = ts.p; g.a = no_img(); g.n2 = no_img();
+    g.colsq_off = ts.colsq;
+    g.out.normal = dest_none(); g.out.normal.f32 = Sel{W_R, 0, 0}; g.out.normal.has_f32 = 1;
+    g.out.normal.img = ts.r; g.out.normal.colsq = 1;
+    g.out.shifted = g.out.normal; g.out.ld = r;
+    if (g_bf16) launch_gemm<tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 1>(b, g, prof::S_K3, st);
+    else launch_gemm<tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K3, st);
 }
 
-// Gram = src^T src (src: rows x r)
-inline void tensor_gram(int64_t, int64_t, int r, int passes, const Batch& b, const TensorScratch& ts, Sel src,
-                        int64_t rows, Sel gram, int only_shift_bit, cudaStream_t st) {
-    const int terms = passes == 3 ? 2 : 1;
-    tc::PackRef sp = make_pack(ts.src_t, r, rows, terms);
-    launch_pack(b, src, rows, r, 1, sp, only_shift_bit, st, ts.colsq);
+// Gram = src^T src (src: image of a rows x r matrix); only tiles that touch the lower triangle
+inline void tensor_gram(int r, int passes, const Batch& b, ImgRef src, int64_t rows, Sel gram, int only_shift_bit,
+                        cudaStream_t st) {
     tc::GemmArgs g{};
-    g.Mrows = r; g.Ncols = r; g.Kdim = (int32_t)rows; g.BN = tensor_bn(r);
-    g.passes = passes; g.passes2 = 1; g.a = sp; g.b = sp;
-    g.st = EpStore{gram, gram, only_shift_bit, 1, r, only_shift_bit ? 1 : 0};
-    launch_gemm<tc::A_PACKED, tc::EPI_STORE>(b, g, prof::S_GRAM, st);
+    g.Mrows = r; g.Ncols = r; g.Kdim = (int32_t)rows; g.BN = std::min(r, 256);
+    g.passes = passes; g.passes2 = 1; g.a = src; g.n1 = src; g.n2 = no_img(); g.lower_only = 1;
+    g.out.normal = dest_none(); g.out.normal.f32 = gram; g.out.normal.has_f32 = 1;
+    g.out.shifted = g.out.normal; g.out.ld = r;
+    g.out.shift_bit = only_shift_bit; g.out.only_if_shifted = only_shift_bit ? 1 : 0;
+    launch_gemm<tc::A_IMG_MN, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_GRAM, st);
 }
 
-// dst = src * L^{-T}  (src: rows x r, L^{-1} lower triangular r x r)
-inline void tensor_apply(int64_t, int64_t, int r, int passes, const Batch& b, const TensorScratch& ts, Sel src,
-                         int64_t rows, Sel linv, EpStore ep, cudaStream_t st) {
-    const int terms = passes == 3 ? 2 : 1;
-    tc::PackRef sp = make_pack(ts.src_n, rows, r, terms);
-    tc::PackRef lp = make_pack(ts.linv, r, r, terms);
-    const int only_bit = ep.only_if_shifted ? ep.shift_bit : 0;
-    launch_pack(b, src, rows, r, 0, sp, only_bit, st);
-    launch_pack(b, linv, r, r, 0, lp, only_bit, st);
+// dst = src * L^{-T}  (src: image of a rows x r matrix, L^{-1}: image linv, lower triangular)
+inline void tensor_apply(int r, int passes, const Batch& b, const TensorScratch& ts, ImgRef src, int64_t rows,
+                         tc::OutSpec out, cudaStream_t st) {
     tc::GemmArgs g{};
-    g.Mrows = (int32_t)rows; g.Ncols = r; g.Kdim = r; g.BN = tensor_bn(r);
-    g.passes = passes; g.passes2 = 1; g.a = sp; g.b = lp; g.tri = 1;
-    g.st = ep;
-    launch_gemm<tc::A_PACKED, tc::EPI_STORE>(b, g, prof::S_APPLY, st);
+    g.Mrows = (int32_t)rows; g.Ncols = r; g.Kdim = r; g.BN = std::min(r, 256);
+    g.passes = passes; g.passes2 = 1; g.a = src; g.n1 = ts.linv; g.n2 = no_img(); g.tri = 1;
+    g.colsq_off = ts.colsq;
+    g.out = out;
+    launch_gemm<tc::A_IMG_K, tc::N_IMG_K, tc::EPI_STORE, 0>(b, g, prof::S_APPLY, st);
 }
 
 // M <- a (M + G) - b P R^T ;  X <- c X - d P Q^T                  (Alg. 1 lines 5-7)
 inline void tensor_k5(int64_t m, int64_t n, int r, int g_bf16, int x_bf16, int passes_m, int passes_x, float ef_a,
                       float ef_b, float wc, float wd, const Batch& b, const TensorScratch& ts, cudaStream_t st) {
-    const int pterms = (passes_m == 3 || passes_x == 3) ? 2 : 1;
-    tc::PackRef pp = make_pack(ts.p_n, m, r, pterms);
-    tc::PackRef rp = make_pack(ts.r_n, n, r, passes_m == 3 ? 2 : 1);
-    tc::PackRef qp = make_pack(ts.q_n, n, r, passes_x == 3 ? 2 : 1);
-    launch_pack(b, Sel{W_P, 0, 0}, m, r, 0, pp, 0, st);
-    launch_pack(b, Sel{W_R, 0, 0}, n, r, 0, rp, 0, st);
-    launch_pack(b, Sel{W_Q, 0, 0}, n, r, 0, qp, 0, st);
     tc::GemmArgs g{};
     g.Mrows = (int32_t)m; g.Ncols = (int32_t)n; g.Kdim = r; g.BN = 128;
-    g.passes = passes_m; g.passes2 = passes_x; g.g_bf16 = g_bf16; g.x_bf16 = x_bf16; g.ld = n;
-    g.a = pp; g.b = rp; g.b2 = qp;
+    g.passes = passes_m; g.passes2 = passes_x; g.ld = n;
+    g.a = ts.p; g.n1 = ts.r; g.n2 = ts.q;
     g.ef_a = ef_a; g.ef_b = ef_b; g.wc = wc; g.wd = wd;
-    launch_gemm<tc::A_PACKED, tc::EPI_K5>(b, g, prof::S_K5, st);
+    g.out.normal = dest_none(); g.out.shifted = dest_none();
+    const int xg = (g_bf16 ? 1 : 0) | (x_bf16 ? 2 : 0);
+    switch (xg) {
+        case 0: launch_gemm<tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 0>(b, g, prof::S_K5, st); break;
+        case 1: launch_gemm<tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 1>(b, g, prof::S_K5, st); break;
+        case 2: launch_gemm<tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 2>(b, g, prof::S_K5, st); break;
+        default: launch_gemm<tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 3>(b, g, prof::S_K5, st); break;
+    }
 }
 
 }  // namespace od
