@@ -221,6 +221,9 @@ def run_ours(args):
             od.orthdion_set_dtypes(h, spec.x_dtype, spec.g_dtype)
             if args.engine == "simt":
                 od.orthdion_set_engine(h, od.ENGINE_SIMT)
+            if args.passes:
+                for which, pv in enumerate(int(x) for x in args.passes.split(",")):
+                    od.orthdion_set_passes(h, which, pv)
             plan_cache[key] = h
         hs.append(plan_cache[key])
         X, M, Q = wl.initial_state(spec, seed, i, device=dev)
@@ -423,6 +426,8 @@ def main():
     ap.add_argument("--rank", type=int, default=None, help="override r (cfg2 sweep)")
     ap.add_argument("--mode", default="orth", choices=["orth", "colnorm"])
     ap.add_argument("--engine", default="tensor", choices=["tensor", "simt"])
+    ap.add_argument("--passes", default=None,
+                    help="bf16 split passes of the four product groups, e.g. 3,3,3,1 (0 keeps the default)")
     ap.add_argument("--grad-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")

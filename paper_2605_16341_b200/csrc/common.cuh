@@ -29,6 +29,7 @@ constexpr int MAXB = 256;   // matrices per launch batch
 struct Batch {
     int32_t count;
     int32_t pad;
+    int64_t scratch_stride;   // w[k].scratch = w[0].scratch + k * scratch_stride (one class per batch)
     MatWork w[MAXB];
 };
 

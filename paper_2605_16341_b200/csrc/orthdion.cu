@@ -184,7 +184,7 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
         if (lead.tensor()) {
             ca.colsq = sel(W_SCRATCH, lead.sc.ts.colsq); ca.use_colsq = 1; ca.img = lead.sc.ts.linv;
         }
-        merged->count = 0; merged->pad = 0;
+        merged->count = 0; merged->pad = 0; merged->scratch_stride = 0;
         auto flush = [&]() {
             if (!merged->count) return;
             prof::Scope scope(prof::S_CHOL, st);
@@ -452,6 +452,7 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
             ClassRun c{hs[idx[0]], &pool[bi], scratch_layout(hs[idx[0]])};
             c.b->count = (int32_t)idx.size();
             c.b->pad = 0;
+            c.b->scratch_stride = (int64_t)c.sc.bytes;
             for (size_t k = 0; k < idx.size(); ++k) {
                 const int i = idx[k];
                 MatWork& w = c.b->w[k];
@@ -464,7 +465,13 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
             }
             cls.push_back(c);
         }
+        engine_error() = 0;
         run_group(cls, merged, st);
+        if (engine_error()) {
+            std::fprintf(stderr, "orthdion: tensor map setup failed (%d)\n", engine_error());
+            rc = ORTHDION_ERR_CUDA;
+            break;
+        }
         cudaError_t ce = cudaGetLastError();
         if (ce != cudaSuccess) {
             std::fprintf(stderr, "orthdion: launch failed: %s\n", cudaGetErrorString(ce));

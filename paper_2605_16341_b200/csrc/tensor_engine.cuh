@@ -4,9 +4,10 @@
 // means t0*u0 + t0*u1 + t1*u0 (relative error about 2^-16), "1 pass" t0*u0.
 //
 // Operands.  Every small operand (Q, Y, P, R, L^{-1} and the QR intermediates) lives in global
-// memory as a split image (common.cuh): ready-made swizzled shared-memory tiles that bulk
-// asynchronous copies (TMA engine, cp.async.bulk) drop into an operand ring, usable both K-major
-// and MN-major, so no kernel ever transposes.  Images are written by the epilogue of the kernel
+// memory as a split image (common.cuh): ready-made swizzled shared-memory tiles that one tiled
+// TMA load (cp.async.bulk.tensor over a 5-d tensor map: 64 elements, rows, panels, terms,
+// matrices of the launch batch) drops into an operand ring, usable both K-major and MN-major,
+// so no kernel ever transposes.  Images are written by the epilogue of the kernel
 // that produces the matrix; only Q_prev (caller-owned fp32) is packed by a kernel of its own.
 // The big operand B = M + G (Alg. 1 line 1) is never stored: transform warps read M and G from
 // HBM, add, split and write the A tile directly.
@@ -15,7 +16,10 @@
 // 32 KB) and N-side pieces (a slice of the other operand, at most 48 KB), each with full/empty
 // mbarriers; accumulators (up to 128 x 512 fp32) sit in tensor memory.
 #pragma once
+#include <cuda.h>
+
 #include <algorithm>
+#include <cstdio>
 
 #include "common.cuh"
 #include "profile.cuh"
@@ -75,6 +79,11 @@ struct GemmArgs {
     int64_t colsq_off;                       // scratch offset of the column-square partials
     float ef_a, ef_b, wc, wd;
     OutSpec out;
+    // tensor maps of the images a, n1, n2 over the whole launch batch; the box of each map is the
+    // tile or piece this launch loads with one instruction
+    alignas(64) CUtensorMap map_a;
+    alignas(64) CUtensorMap map_n1;
+    alignas(64) CUtensorMap map_n2;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -114,9 +123,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+// One tiled TMA load: the box of `map` at (0, row, panel, term 0, matrix) -> shared memory, laid
+// out [term][panel][row][128 bytes]; completes on the mbarrier with the full box size.
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int row, int panel, int matrix,
+                                             uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(panel), "r"(0), "r"(matrix), "r"(bar)
+        : "memory");
+}
+// Hint: bring the line at p into L2.
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 __device__ __forceinline__ void fence_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -334,71 +352,84 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
 
     const int a_terms = (g.passes == 3 || (EPI == EPI_K5 && g.passes2 == 3)) ? 2 : 1;
     const int n1_terms = g.passes == 3 ? 2 : 1;
-    const int n2_terms = g.passes2 == 3 ? 2 : 1;
     // N_IMG_MN piece geometry: [term][64-column group][ks rows of 128 bytes]
     const uint32_t group_stride = (uint32_t)g.ks * 128u;
     const uint32_t mn_term_stride = (uint32_t)((g.BN + 63) / 64) * group_stride;
 
     if (warp == 0) {
         // ---------------- producer ----------------
-        if (lane == 0) {
+        // Lane 0 arms the barrier of a slot and issues the one TMA load that fills it.  For the
+        // fused feedback/update pass the whole warp also asks for the next tile's M, G, X in L2,
+        // so that the epilogue's loads see L2 latency and need few bytes in flight.
+        {
             int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
             bool ok = true;
+            constexpr int GB = G_BF16 ? 2 : 4, XB = X_BF16 ? 2 : 4;
+            auto prefetch_k5 = [&](int t) {
+                if (t >= g.total_tiles) return;
+                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                if (!c.active) return;
+                const MatWork& w = batch.w[c.b];
+                const int ncols = min(g.BN, g.Ncols - c.n0);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int64_t gi = (int64_t)c.mt * BM + lane + 32 * i;
+                    if (gi < g.Mrows) {
+                        const int64_t off = gi * g.ld + c.n0;
+                        const char* pm = reinterpret_cast<const char*>(w.M + off);
+                        const char* pg = reinterpret_cast<const char*>(w.G) + off * GB;
+                        const char* px = reinterpret_cast<const char*>(w.X) + off * XB;
+                        for (int o = 0; o < ncols * 4; o += 64) prefetch_l2(pm + o);
+                        for (int o = 0; o < ncols * GB; o += 64) prefetch_l2(pg + o);
+                        for (int o = 0; o < ncols * XB; o += 64) prefetch_l2(px + o);
+                    }
+                }
+            };
+            if (EPI == EPI_K5) prefetch_k5(blockIdx.x);
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
                 const TileCoord c = decode_tile<EPI>(batch, g, t);
+                if (EPI == EPI_K5) prefetch_k5(t + gridDim.x);
                 if (!c.active) continue;
-                const unsigned char* scr = reinterpret_cast<const unsigned char*>(batch.w[c.b].scratch);
                 for (int kb = 0; kb < c.kb_end && ok; ++kb) {
                     if (!A_BUF) {
-                        if (!mbar_wait(a_empty0 + 8 * as, aph ^ 1, abort_flag)) { ok = false; break; }
-                        const uint32_t fb = a_full0 + 8 * as;
-                        const uint32_t dst = smem_u32(a_ring + as * A_SLOT_BYTES);
-                        if (AMODE == A_IMG_K) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(a_empty0 + 8 * as, aph ^ 1, abort_flag));
+                        if (!ok) break;
+                        if (lane == 0) {
+                            const uint32_t fb = a_full0 + 8 * as;
+                            const uint32_t dst = smem_u32(a_ring + as * A_SLOT_BYTES);
                             mbar_arrive_expect_tx(fb, (uint32_t)a_terms * A_TERM_BYTES);
-                            for (int term = 0; term < a_terms; ++term)
-                                bulk_copy_g2s(dst + term * A_TERM_BYTES,
-                                              scr + img_row_offset(g.a, term, kb, (int64_t)c.mt * BM), A_TERM_BYTES, fb);
-                        } else {
-                            const int ng = min(2, g.a.panels - c.mt * 2);
-                            mbar_arrive_expect_tx(fb, (uint32_t)(a_terms * ng) * 8192u);
-                            for (int term = 0; term < a_terms; ++term)
-                                for (int gi = 0; gi < ng; ++gi)
-                                    bulk_copy_g2s(dst + term * A_TERM_BYTES + gi * 8192,
-                                                  scr + img_row_offset(g.a, term, c.mt * 2 + gi, (int64_t)kb * BK), 8192, fb);
+                            if (AMODE == A_IMG_K) tma_load_box(dst, &g.map_a, c.mt * BM, kb, c.b, fb);
+                            else tma_load_box(dst, &g.map_a, kb * BK, c.mt * 2, c.b, fb);
                         }
                         if (++as == A_SLOTS) { as = 0; aph ^= 1; }
                     }
                     if (NMODE == N_IMG_MN) {
                         const int pieces = mn_pieces(g, kb);
-                        const int np = (c.bn + 63) / 64, p0 = c.n0 / 64;
                         for (int sub = 0; sub < pieces && ok; ++sub) {
-                            if (!mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag)) { ok = false; break; }
-                            const uint32_t fb = n_full0 + 8 * ns;
-                            const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
-                            mbar_arrive_expect_tx(fb, (uint32_t)(n1_terms * np) * group_stride);
-                            for (int term = 0; term < n1_terms; ++term)
-                                for (int i = 0; i < np; ++i)
-                                    bulk_copy_g2s(dst + term * mn_term_stride + i * group_stride,
-                                                  scr + img_row_offset(g.n1, term, p0 + i, (int64_t)kb * BK + sub * g.ks),
-                                                  group_stride, fb);
+                            ok = __all_sync(0xffffffffu, mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag));
+                            if (!ok) break;
+                            if (lane == 0) {
+                                const uint32_t fb = n_full0 + 8 * ns;
+                                mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
+                                tma_load_box(smem_u32(n_ring + (size_t)ns * g.n_piece_bytes), &g.map_n1,
+                                             kb * BK + sub * g.ks, c.n0 / 64, c.b, fb);
+                            }
                             if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
                         }
                     } else {
                         const int chunks = (c.bn + 127) / 128;
                         for (int ch = 0; ch < chunks && ok; ++ch) {
                             if (!k_piece_active(g, c, kb, ch)) continue;
-                            if (!mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag)) { ok = false; break; }
-                            const uint32_t fb = n_full0 + 8 * ns;
-                            const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
-                            const int nt_all = n1_terms + (EPI == EPI_K5 ? n2_terms : 0);
-                            mbar_arrive_expect_tx(fb, (uint32_t)nt_all * A_TERM_BYTES);
-                            for (int term = 0; term < n1_terms; ++term)
-                                bulk_copy_g2s(dst + term * A_TERM_BYTES,
-                                              scr + img_row_offset(g.n1, term, kb, (int64_t)c.n0 + ch * 128), A_TERM_BYTES, fb);
-                            if (EPI == EPI_K5)
-                                for (int term = 0; term < n2_terms; ++term)
-                                    bulk_copy_g2s(dst + (n1_terms + term) * A_TERM_BYTES,
-                                                  scr + img_row_offset(g.n2, term, kb, (int64_t)c.n0 + ch * 128), A_TERM_BYTES, fb);
+                            ok = __all_sync(0xffffffffu, mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag));
+                            if (!ok) break;
+                            if (lane == 0) {
+                                const uint32_t fb = n_full0 + 8 * ns;
+                                const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                                mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
+                                tma_load_box(dst, &g.map_n1, c.n0 + ch * 128, kb, c.b, fb);
+                                if (EPI == EPI_K5)
+                                    tma_load_box(dst + n1_terms * A_TERM_BYTES, &g.map_n2, c.n0 + ch * 128, kb, c.b, fb);
+                            }
                             if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
                         }
                     }
@@ -593,9 +624,8 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             // Fused error feedback and weight update.  Warp (quarter, half) owns rows
             // 32*quarter.. of the tile and columns 64*half.., in two slabs of 32 x 32.  The two
             // accumulator slabs go through a swizzled staging block so that global accesses run
-            // along rows (8 lanes x 16 bytes per row); M, G, X of the next slab are fetched
-            // before the current one is finished.
-            constexpr bool PF = G_BF16 && X_BF16;
+            // along rows (8 lanes x 16 bytes per row).  The producer warp has already asked for the
+            // tile's M, G, X in L2, so the loads of a slab return with L2 latency.
             const int half = (warp - 2) / 4;
             unsigned char* S1 = staging + (warp - 2) * STAGING_BYTES_PER_WARP;
             unsigned char* S2 = S1 + 4096;
@@ -634,40 +664,31 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 }
             };
 
-            K5Pre<XG> pre, cur;
-            int t = blockIdx.x - (int)gridDim.x;
-            t = next_tile(t);
-            int slab = 0;
-            if (PF && t < g.total_tiles) fetch(pre, t, 0);
-            while (t < g.total_tiles && ok) {
-                int t2 = t, slab2 = slab + 1;
-                if (slab2 == 2) { slab2 = 0; t2 = next_tile(t); }
-                if constexpr (PF) {
-                    cur = pre;
-                    if (t2 < g.total_tiles) fetch(pre, t2, slab2);
-                } else {
-                    fetch(cur, t, slab);
-                }
+            // one slab: accumulators -> staging -> row-wise update of M and X
+            auto process = [&](const K5Pre<XG>& cur, int t, int slab) -> bool {
                 const TileCoord c = decode_tile<EPI>(batch, g, t);
                 const MatWork& w = batch.w[c.b];
                 if (slab == 0) {
-                    if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) return false;
                     tc_fence_after();
                 }
                 const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16) +
                                        (uint32_t)(half * 64 + slab * 32);
                 {
-                    uint32_t v1[32], v2[32];
-                    tmem_ld16(taddr, *reinterpret_cast<uint32_t(*)[16]>(&v1[0]));
-                    tmem_ld16(taddr + 16, *reinterpret_cast<uint32_t(*)[16]>(&v1[16]));
-                    tmem_ld16(taddr + g.BN, *reinterpret_cast<uint32_t(*)[16]>(&v2[0]));
-                    tmem_ld16(taddr + g.BN + 16, *reinterpret_cast<uint32_t(*)[16]>(&v2[16]));
+                    uint32_t va[16], vb[16], vc[16], vd[16];
+                    tmem_ld16(taddr, va);
+                    tmem_ld16(taddr + 16, vb);
+                    tmem_ld16(taddr + g.BN, vc);
+                    tmem_ld16(taddr + g.BN + 16, vd);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        const int o = lane * 128 + img_chunk_offset(lane, ch);
-                        *reinterpret_cast<uint4*>(S1 + o) = make_uint4(v1[4 * ch], v1[4 * ch + 1], v1[4 * ch + 2], v1[4 * ch + 3]);
-                        *reinterpret_cast<uint4*>(S2 + o) = make_uint4(v2[4 * ch], v2[4 * ch + 1], v2[4 * ch + 2], v2[4 * ch + 3]);
+                    for (int ch = 0; ch < 4; ++ch) {
+                        const int o0 = lane * 128 + img_chunk_offset(lane, ch);
+                        const int o1 = lane * 128 + img_chunk_offset(lane, ch + 4);
+                        *reinterpret_cast<uint4*>(S1 + o0) = make_uint4(va[4 * ch], va[4 * ch + 1], va[4 * ch + 2], va[4 * ch + 3]);
+                        *reinterpret_cast<uint4*>(S1 + o1) = make_uint4(vb[4 * ch], vb[4 * ch + 1], vb[4 * ch + 2], vb[4 * ch + 3]);
+                        *reinterpret_cast<uint4*>(S2 + o0) = make_uint4(vc[4 * ch], vc[4 * ch + 1], vc[4 * ch + 2], vc[4 * ch + 3]);
+                        *reinterpret_cast<uint4*>(S2 + o1) = make_uint4(vd[4 * ch], vd[4 * ch + 1], vd[4 * ch + 2], vd[4 * ch + 3]);
                     }
                 }
                 __syncwarp();
@@ -723,7 +744,19 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                     if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
                     if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
                 }
-                t = t2; slab = slab2;
+                return true;
+            };
+            // the slabs of this warp in order: (tile, 0), (tile, 1), (next tile, 0), ...
+            auto advance = [&](int& t, int& slab) {
+                if (++slab == 2) { slab = 0; t = next_tile(t); }
+            };
+
+            int t = next_tile(blockIdx.x - (int)gridDim.x), slab = 0;
+            K5Pre<XG> pa;
+            while (t < g.total_tiles) {
+                fetch(pa, t, slab);
+                if (!process(pa, t, slab)) break;
+                advance(t, slab);
             }
         }
     } else if (A_BUF) {
@@ -898,6 +931,49 @@ inline ImgRef img_view(const ImgRef& im, int64_t rows) {
     return v;
 }
 
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link libcuda.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline TensorMapEncodeFn tensor_map_encoder() {
+    static TensorMapEncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<TensorMapEncodeFn>(p);
+    }
+    return fn;
+}
+// First error met while preparing launches of the current step call (0 = none).
+inline int& engine_error() { static int e = 0; return e; }
+
+// 5-d map over the images `img` of all matrices of a batch: (64 bf16, rows, panels, terms, matrix),
+// with the box (64, box_rows, box_panels, box_terms, 1).  The images are stored pre-swizzled, so
+// the copy itself does not swizzle; out-of-range parts of a box read as zeros.
+inline void encode_img_map(CUtensorMap* map, const Batch& b, const ImgRef& img, int box_rows, int box_panels,
+                           int box_terms) {
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (!enc) { engine_error() = 1; return; }
+    const cuuint64_t term_bytes = (cuuint64_t)img.panels * img.rows_pad * 128;
+    cuuint64_t dims[5] = {64, (cuuint64_t)img.rows_pad, (cuuint64_t)img.panels, 2, (cuuint64_t)b.count};
+    cuuint64_t strides[4] = {128, (cuuint64_t)img.rows_pad * 128, term_bytes,
+                             b.count > 1 ? (cuuint64_t)b.scratch_stride : 2 * term_bytes};
+    cuuint32_t box[5] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_panels, (cuuint32_t)box_terms, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    void* base = b.w[0].scratch + img.off;
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        std::fprintf(stderr, "orthdion: cuTensorMapEncodeTiled failed (%d)\n", (int)r);
+        engine_error() = 2;
+    }
+}
+
 inline int sm_count() {
     static int n = 0;
     if (!n) {
@@ -966,6 +1042,13 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     g.n_slots = (int)std::min<size_t>(tc::MAX_N_SLOTS, (tc::SMEM_LIMIT - fixed) / (size_t)g.n_piece_bytes);
     // more than half of an SM's shared memory: one CTA per SM, whatever its tensor-memory share
     const size_t smem = std::max<size_t>(fixed + (size_t)g.n_slots * g.n_piece_bytes, 120 * 1024);
+    const int a_terms = (g.passes == 3 || (EPI == tc::EPI_K5 && g.passes2 == 3)) ? 2 : 1;
+    if (AMODE == tc::A_IMG_K) encode_img_map(&g.map_a, b, g.a, 128, 1, a_terms);
+    else if (AMODE == tc::A_IMG_MN) encode_img_map(&g.map_a, b, g.a, 64, 2, a_terms);
+    if (NMODE == tc::N_IMG_MN) encode_img_map(&g.map_n1, b, g.n1, g.ks, bn64 / 64, n1_terms);
+    else encode_img_map(&g.map_n1, b, g.n1, 128, 1, n1_terms);
+    if (EPI == tc::EPI_K5) encode_img_map(&g.map_n2, b, g.n2, 128, 1, n2_terms);
+    if (engine_error()) return;
     const int grid = std::min(g.total_tiles, sm_count());
     prof::Scope scope(stage, st);
     tc::gemm_kernel<AMODE, NMODE, EPI, XG><<<grid, tc::gemm_threads(AMODE, EPI), smem, st>>>(b, g);
