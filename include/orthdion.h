@@ -111,6 +111,33 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count,
                           void* const* X, float* const* M, const void* const* G, float* const* Q,
                           void* workspace, size_t workspace_bytes, void* stream);
 
+/* One step for one matrix without any caller-provided workspace and without any device-memory
+ * allocation.  (The paper has no counterpart: this entry point exists for the integration, not
+ * for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region that is being
+ * stream-captured, inside a framework callback that must not touch the allocator, or in a process
+ * whose memory pool was sized up front and locked.  Such a caller cannot size and allocate the
+ * workspace that orthdion_step asks for, so here the scratch lives in a fixed array that is part
+ * of the library image itself: ORTHDION_NOALLOC_SCRATCH_BYTES bytes of device memory on every
+ * GPU that loads the library, held until the process exits.
+ *
+ *  - X, M, G, Q: as for orthdion_step (device pointers, updated in place, G read only).
+ *  - status_dev: optional DEVICE pointer to one int32; when not null the matrix's status flags
+ *    (ORTHDION_STATUS_*) are copied there in stream order.  The factors P and R are not exposed.
+ *  - A plan whose orthdion_workspace_bytes() exceeds ORTHDION_NOALLOC_SCRATCH_BYTES is rejected
+ *    with ORTHDION_ERR_WORKSPACE (and a message on stderr); nothing is enqueued then.
+ *  - The first call on a device looks up the device address of the array (no allocation).  Make
+ *    that first call outside of any stream capture.
+ *  - All calls share the one array, and it keeps whatever the previous call left in it; the step
+ *    rewrites everything it later reads.  Two calls whose kernels overlap on the GPU (different
+ *    streams, or several host threads) race on it: keep calls on one stream, or order them.
+ *  - Results are those of orthdion_step on the same inputs.  Host-side bookkeeping may use the
+ *    host heap; no CUDA allocation routine is called. */
+#define ORTHDION_NOALLOC_SCRATCH_BYTES ((size_t)64 << 20)
+int orthdion_step_noalloc(orthdion_t h, void* X, float* M, const void* G, float* Q,
+                          int32_t* status_dev, void* stream);
+
 /* Device pointers to the factors P (m x r) and R (n x r) that the last step left in the
  * workspace (for checks).  index = position in the grouped call, 0 for orthdion_step. */
 int orthdion_get_factors(const orthdion_t* hs, int32_t count, int32_t index, void* workspace,

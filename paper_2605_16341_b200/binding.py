@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
     L.orthdion_workspace_bytes_grouped.restype = sz
     L.orthdion_step.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.orthdion_step_grouped.argtypes = [pvp, i32, pvp, pvp, pvp, pvp, vp, sz, vp]
+    L.orthdion_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.orthdion_get_factors.argtypes = [pvp, i32, i32, vp, pvp, pvp]
     L.orthdion_last_status.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(i32)]
     L.orthdion_version.restype = ctypes.c_char_p
@@ -86,7 +87,7 @@ def lib() -> ctypes.CDLL:
     L.orthdion_stage_name.argtypes = [i32]
     L.orthdion_stage_name.restype = ctypes.c_char_p
     for name in ("create", "destroy", "set_dtypes", "set_lr", "set_scale", "set_ef", "set_engine",
-                 "set_passes", "step", "step_grouped", "get_factors", "last_status"):
+                 "set_passes", "step", "step_grouped", "step_noalloc", "get_factors", "last_status"):
         getattr(L, "orthdion_" + name).restype = i32
     _lib = L
     return L
@@ -95,7 +96,7 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ["orthdion_create", "orthdion_destroy", "orthdion_set_dtypes", "orthdion_set_lr",
             "orthdion_set_scale", "orthdion_set_ef", "orthdion_set_engine", "orthdion_set_passes",
             "orthdion_workspace_bytes", "orthdion_workspace_bytes_grouped", "orthdion_step",
-            "orthdion_step_grouped", "orthdion_get_factors", "orthdion_last_status", "orthdion_version",
+            "orthdion_step_grouped", "orthdion_step_noalloc", "orthdion_get_factors", "orthdion_last_status", "orthdion_version",
             "orthdion_launch_count", "orthdion_profile_begin", "orthdion_profile_end", "orthdion_stage_count",
             "orthdion_stage_name"]
 
@@ -180,6 +181,21 @@ def orthdion_step(h, X, M, G, Q, workspace, stream=None):
     _check(lib().orthdion_step(h, _dev_ptr(X, "X"), _dev_ptr(M, "M"), _dev_ptr(G, "G"), _dev_ptr(Q, "Q"),
                                _dev_ptr(workspace, "workspace"), workspace.numel() * workspace.element_size(),
                                _stream_ptr(stream)), "orthdion_step")
+
+
+NOALLOC_SCRATCH_BYTES = 64 << 20
+
+
+def orthdion_step_noalloc(h, X, M, G, Q, status=None, stream=None):
+    """One step for one matrix with the library's built-in scratch array: no workspace argument
+    and no device allocation anywhere in the call (for callers that must not allocate, e.g. while
+    a stream is being captured or when the memory pool is locked).  `status`, if given, is a
+    one-element int32 CUDA tensor that receives the status flags in stream order.  Plans that
+    need more than NOALLOC_SCRATCH_BYTES are rejected (OrthDionError WORKSPACE).  Calls share
+    the array: do not let two of them overlap on the GPU."""
+    sp = 0 if status is None else _dev_ptr(status, "status")
+    _check(lib().orthdion_step_noalloc(h, _dev_ptr(X, "X"), _dev_ptr(M, "M"), _dev_ptr(G, "G"), _dev_ptr(Q, "Q"),
+                                       sp, _stream_ptr(stream)), "orthdion_step_noalloc")
 
 
 class PointerTable:

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -489,6 +490,61 @@ int orthdion_step(orthdion_t h, void* X, float* M, const void* G, float* Q, void
     const void* const gs[1] = {G};
     float* const qs[1] = {Q};
     return orthdion_step_grouped(&h, 1, xs, ms, gs, qs, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+// Scratch of orthdion_step_noalloc: part of the library image, so every GPU that loads the library
+// holds these bytes until the process exits.  In host code the name below is only a handle for
+// cudaGetSymbolAddress; it is not a device address and must never be handed to a kernel.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ORTHDION_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+// Device address of g_noalloc_scratch on the current device, looked up once per device.
+int noalloc_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* addr[kMaxDevices] = {};
+    int dev = -1;
+    CU_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return ORTHDION_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        CU_CHECK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (!p) return ORTHDION_ERR_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return ORTHDION_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int orthdion_step_noalloc(orthdion_t h, void* X, float* M, const void* G, float* Q, int32_t* status_dev,
+                          void* stream) {
+    if (!valid(h)) return ORTHDION_ERR_INVALID_ARG;
+    const size_t need = orthdion_workspace_bytes(h);
+    if (need == 0) return ORTHDION_ERR_INVALID_ARG;
+    if (need > ORTHDION_NOALLOC_SCRATCH_BYTES) {
+        std::fprintf(stderr,
+                     "orthdion_step_noalloc: this plan (m=%lld, n=%lld, r=%d) needs %zu bytes of scratch, the "
+                     "built-in array holds %zu; use orthdion_step with a caller-provided workspace\n",
+                     (long long)h->m, (long long)h->n, (int)h->r, need, (size_t)ORTHDION_NOALLOC_SCRATCH_BYTES);
+        return ORTHDION_ERR_WORKSPACE;
+    }
+    void* scratch = nullptr;
+    int rc = noalloc_scratch_address(&scratch);
+    if (rc) return rc;
+    rc = orthdion_step(h, X, M, G, Q, scratch, ORTHDION_NOALLOC_SCRATCH_BYTES, stream);
+    if (rc) return rc;
+    if (status_dev) {
+        // the status word of the only matrix is the first word of the scratch
+        CU_CHECK(cudaMemcpyAsync(status_dev, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice,
+                                 reinterpret_cast<cudaStream_t>(stream)));
+    }
+    return ORTHDION_OK;
 }
 
 int orthdion_get_factors(const orthdion_t* hs, int32_t count, int32_t index, void* workspace,
