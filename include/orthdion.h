@@ -90,9 +90,12 @@ int orthdion_set_lr(orthdion_t h, float eta);               /* eta_t of a schedu
 int orthdion_set_scale(orthdion_t h, float scale);          /* extra factor on the update; 1.0   */
 int orthdion_set_ef(orthdion_t h, float a, float b);        /* M <- a*B - b*P*R^T                */
 int orthdion_set_engine(orthdion_t h, int32_t engine);
-/* Number of bf16 split terms products are built from (1 = plain bf16, 3 = three products of a
- * two-term split, about 2^-16 relative accuracy).  which: 0 = B*Q and B^T*P, 1 = Gram/apply of
- * the QR, 2 = P*R^T of the error feedback, 3 = P*Q^T of the weight update. <=0 restores default. */
+/* Number of tensor-core passes products are built from (3 = three bf16 products of a two-term
+ * split, about 2^-16 relative accuracy; 1 = one pass).  which: 0 = B*Q and B^T*P, 1 = Gram/apply
+ * of the QR, 2 = P*R^T of the error feedback, 3 = P*Q^T of the weight update.  When both 2 and 3
+ * ask for one pass, the fused pass runs in fp16 (11-bit operands, R scaled by a power of two);
+ * otherwise a single pass means plain bf16.  Defaults: 3, 3, and 1, 1 for bf16 weights (3, 3 for
+ * fp32 weights).  passes <= 0 restores the default. */
 int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes);
 
 /* Workspace sizes in bytes (host computation, no CUDA call). */

@@ -67,6 +67,18 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t p) { return __uint_as_float(p & 0xFFFF0000u); }
 
+// two fp32 -> packed f16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// 8 fp32 values (times scale) -> 16-byte chunk of fp16
+__device__ __forceinline__ uint4 half8(const float (&v)[8], float scale) {
+    return make_uint4(pack_f16x2(v[0] * scale, v[1] * scale), pack_f16x2(v[2] * scale, v[3] * scale),
+                      pack_f16x2(v[4] * scale, v[5] * scale), pack_f16x2(v[6] * scale, v[7] * scale));
+}
+
 // 8 fp32 values -> 16-byte chunk of term 0 and of term 1
 __device__ __forceinline__ void split8(const float (&v)[8], uint4& t0, uint4& t1) {
     uint32_t a[4], b[4];
@@ -88,10 +100,14 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4& t0, uint4& t1
 // of panel p starts at off + (t * panels + p) * rows_pad * 128.  128 consecutive rows of a panel
 // are a K-major operand tile (depth = S columns); 64 consecutive rows of two or more panels are an
 // MN-major operand tile (depth = S rows): bulk copies move either into shared memory unchanged.
+// An image may carry a third plane (index 2): the matrix rounded once to fp16 (times a power of
+// two chosen by the writer), for products that run as a single fp16 pass.
 struct ImgRef {
     int64_t off;        // byte offset in the matrix's scratch area; < 0: absent
     int32_t rows_pad;   // multiple of 128
     int32_t panels;     // ceil(cols / 64)
+    int32_t planes;     // 2 (bf16 terms) or 3 (+ fp16 plane)
+    int32_t pad;
 };
 __device__ __forceinline__ int64_t img_row_offset(const ImgRef& im, int term, int panel, int64_t row) {
     return im.off + (((int64_t)term * im.panels + panel) * im.rows_pad + row) * 128;

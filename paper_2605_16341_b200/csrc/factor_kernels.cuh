@@ -78,6 +78,7 @@ struct CholArgs {
     Sel colsq;
     int32_t use_colsq, pad;
     ImgRef img;      // img.off >= 0: also write L^{-1} as a split image (tensor-core operand)
+    int64_t cnorm_off;   // >= 0: also leave the Gram diagonal (squared column norms) there, fp32 [r]
 };
 
 // Factor Gram = L L^T (blocked, right-looking) and overwrite `work` with L^{-1}.
@@ -124,6 +125,7 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
                 d = A[(int64_t)i * r + i];
             }
             s_diag[i] = d;
+            if (a.cnorm_off >= 0) reinterpret_cast<float*>(w.scratch + a.cnorm_off)[i] = d;
             t += d;
         }
         for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -351,7 +353,7 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
 // ---- ColNorm (Alg. 1 line 4, Dion branch): Q[:,j] = R[:,j] / ||R[:,j]||_2 ----------------------
 // One CTA per 32 columns: 32 x 32 threads, lanes along columns (coalesced rows).
 __global__ void __launch_bounds__(1024)
-colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r) {
+colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t cnorm_off) {
     const MatWork& w = batch.w[blockIdx.z];
     if (*w.status & ST_FAILED) return;
     __shared__ float part[32][33];
@@ -366,6 +368,7 @@ colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r) {
     if (ry == 0) {
         float t = 0.f;
         for (int k = 0; k < 32; ++k) t += part[k][lane];
+        if (cnorm_off >= 0 && j < r) reinterpret_cast<float*>(w.scratch + cnorm_off)[j] = t;
         float nrm = sqrtf(t);
         if (j < r && !(nrm > 0.f)) atomicOr(w.status, ST_ZEROCOL);
         inv[lane] = (nrm > 0.f) ? 1.f / nrm : 0.f;

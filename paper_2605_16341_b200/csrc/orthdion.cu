@@ -51,6 +51,11 @@ struct Scratch {
     size_t bytes;
 };
 
+// The fused feedback/update pass runs as one fp16 pass when both of its products ask for one pass.
+bool fused_fp16(const orthdion_plan* p) {
+    return p->engine == ORTHDION_ENGINE_TENSOR && p->passes[2] == 1 && p->passes[3] == 1;
+}
+
 Scratch scratch_layout(const orthdion_plan* p) {
     Scratch s{};
     const size_t rr = align_up((size_t)p->r * p->r * 4, 256);
@@ -58,7 +63,7 @@ Scratch scratch_layout(const orthdion_plan* p) {
     s.gram = off; off += rr;
     s.linv = off; off += rr;
     if (p->engine == ORTHDION_ENGINE_TENSOR) {
-        off = tensor_scratch_layout(p->m, p->n, p->r, off, &s.ts);
+        off = tensor_scratch_layout(p->m, p->n, p->r, fused_fp16(p), off, &s.ts);
     } else {
         const size_t kr = align_up((size_t)std::max(p->m, p->n) * p->r * 4, 256);
         s.tmpA = off; off += kr;
@@ -181,9 +186,10 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
         CholArgs ca{};
         ca.gram = sel(W_SCRATCH, lead.sc.gram); ca.work = sel(W_SCRATCH, lead.sc.linv);
         ca.r = r; ca.which = which; ca.pass = pass; ca.shift_rel = kShiftRel; ca.cond_limit = kCondLimit;
-        ca.colsq = sel(W_SCRATCH, 0); ca.use_colsq = 0; ca.img = no_img();
+        ca.colsq = sel(W_SCRATCH, 0); ca.use_colsq = 0; ca.img = no_img(); ca.cnorm_off = -1;
         if (lead.tensor()) {
             ca.colsq = sel(W_SCRATCH, lead.sc.ts.colsq); ca.use_colsq = 1; ca.img = lead.sc.ts.linv;
+            if (which == 1 && pass == 1) ca.cnorm_off = lead.sc.ts.cnorm;
         }
         merged->count = 0; merged->pad = 0; merged->scratch_stride = 0;
         auto flush = [&]() {
@@ -306,7 +312,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
         {
             dim3 grid((unsigned)((p->r + 31) / 32), 1, (unsigned)c.b->count);
             prof::Scope scope(prof::S_COLNORM, st);
-            colnorm_kernel<<<grid, 1024, 0, st>>>(*c.b, p->n, p->r);
+            colnorm_kernel<<<grid, 1024, 0, st>>>(*c.b, p->n, p->r, c.tensor() ? c.sc.ts.cnorm : (int64_t)-1);
         }
         if (c.tensor()) launch_pack(*c.b, sQ, p->n, p->r, c.sc.ts.q, st);
     }
@@ -316,7 +322,10 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
         const int gb = p->g_dtype == ORTHDION_DTYPE_BF16, xb = p->x_dtype == ORTHDION_DTYPE_BF16;
         const float cc = 1.f - p->eta * p->wd, dd = p->eta * p->scale;
         if (c.tensor()) {
-            tensor_k5(p->m, p->n, p->r, gb, xb, p->passes[2], p->passes[3], p->ef_a, p->ef_b, cc, dd, *c.b, c.sc.ts, st);
+            const int fp16 = fused_fp16(p) ? 1 : 0;
+            if (fp16) launch_pack_half(*c.b, p->n, p->r, c.sc.ts, st);
+            tensor_k5(p->m, p->n, p->r, gb, xb, p->passes[2], p->passes[3], fp16, p->ef_a, p->ef_b, cc, dd, *c.b,
+                      c.sc.ts, st);
         } else {
             launch_simt(*c.b, p->m, p->n, p->r, RdPlain{sP, p->r, 1}, RdPlain{sR, p->r, 1},
                         EpErrorFeedback{p->ef_a, p->ef_b, p->n, gb}, prof::S_K5, st);
@@ -352,7 +361,7 @@ int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r, float mu, 
     p->mode = mode;
     p->x_dtype = ORTHDION_DTYPE_BF16; p->g_dtype = ORTHDION_DTYPE_BF16;
     p->engine = tensor_engine_supports(m, n, r) ? ORTHDION_ENGINE_TENSOR : ORTHDION_ENGINE_SIMT;
-    p->passes[0] = 3; p->passes[1] = 3; p->passes[2] = 3; p->passes[3] = 1;
+    p->passes[0] = 3; p->passes[1] = 3; p->passes[2] = 1; p->passes[3] = 1;
     *out = p;
     return ORTHDION_OK;
 }
@@ -370,8 +379,10 @@ int orthdion_set_dtypes(orthdion_t h, int32_t x_dtype, int32_t g_dtype) {
         (g_dtype != ORTHDION_DTYPE_F32 && g_dtype != ORTHDION_DTYPE_BF16))
         return ORTHDION_ERR_INVALID_ARG;
     h->x_dtype = x_dtype; h->g_dtype = g_dtype;
-    // an fp32 weight matrix shows the update at full precision: build P Q^T from split terms too
-    h->passes[3] = (x_dtype == ORTHDION_DTYPE_F32) ? 3 : 1;
+    // bf16 weights: the fused feedback/update pass runs as one fp16 pass (11-bit operands: the
+    // feedback term b*P*R^T stays below 1e-5 of the buffer, the update is rounded to bf16 anyway).
+    // An fp32 weight matrix shows the update at full precision: both products from split terms.
+    h->passes[2] = h->passes[3] = (x_dtype == ORTHDION_DTYPE_F32) ? 3 : 1;
     return ORTHDION_OK;
 }
 
@@ -405,7 +416,7 @@ int orthdion_set_engine(orthdion_t h, int32_t engine) {
 int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes) {
     if (!valid(h) || which < 0 || which > 3) return ORTHDION_ERR_INVALID_ARG;
     if (passes <= 0) {
-        passes = (which == 3) ? (h->x_dtype == ORTHDION_DTYPE_F32 ? 3 : 1) : 3;
+        passes = (which >= 2) ? (h->x_dtype == ORTHDION_DTYPE_F32 ? 3 : 1) : 3;
     } else if (passes != 1 && passes != 3) {
         return ORTHDION_ERR_INVALID_ARG;
     }

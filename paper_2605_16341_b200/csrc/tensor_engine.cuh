@@ -31,8 +31,8 @@ namespace tc {
 constexpr int BM = 128;                      // tile rows (MMA M)
 constexpr int BK = 64;                       // depth of one A tile: 64 bf16 = one 128-byte row
 constexpr int A_TERM_BYTES = 128 * 128;      // one 128 x 64 bf16 tile
-constexpr int A_SLOT_BYTES = 2 * A_TERM_BYTES;
-constexpr int A_SLOTS = 2;
+constexpr int A_RING_BYTES = 4 * A_TERM_BYTES;   // two slots of two terms, or four slots of one
+constexpr int MAX_A_SLOTS = 4;
 constexpr int MAX_N_SLOTS = 6;
 constexpr int NUM_XF_WARPS = 16;             // transform warps of the kernels that form B = M + G
 constexpr int STAGING_BYTES_PER_WARP = 8192; // K5 epilogue: two 32 x 32 fp32 blocks per warp
@@ -73,7 +73,10 @@ struct GemmArgs {
     int32_t n_slots, n_piece_bytes;          // N ring
     int32_t acc_bufs;                        // accumulator buffers in tensor memory (1 or 2)
     int32_t tmem_cols;                       // allocation (power of two >= 32)
-    int32_t pad0;
+    int32_t fp16;                            // single-pass fp16 products from plane 2 of the images
+    int32_t a_slots, a_slot_bytes;           // A ring
+    int32_t epi_bufs, pad1;                  // fused pass: 8 KB epilogue buffers per warp (1 or 2)
+    int64_t rscale_off;                      // fp16 fused pass: scratch offset of 1 / (scale of R's plane)
     int64_t ld;                              // leading dimension of M, G, X
     ImgRef a, n1, n2;
     int64_t colsq_off;                       // scratch offset of the column-square partials
@@ -123,19 +126,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
-// One tiled TMA load: the box of `map` at (0, row, panel, term 0, matrix) -> shared memory, laid
+// One tiled TMA load: the box of `map` at (0, row, panel, plane, matrix) -> shared memory, laid
 // out [term][panel][row][128 bytes]; completes on the mbarrier with the full box size.
-__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int row, int panel, int matrix,
-                                             uint32_t bar) {
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int row, int panel, int plane,
+                                             int matrix, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(panel), "r"(0), "r"(matrix), "r"(bar)
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(panel), "r"(plane), "r"(matrix), "r"(bar)
         : "memory");
 }
-// Hint: bring the line at p into L2.
-__device__ __forceinline__ void prefetch_l2(const void* p) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+// Asynchronous 16-byte copy global -> shared (no register staging), grouped per thread.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void fence_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -185,8 +191,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 // Instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = n; a_mn / b_mn = 1 for an
 // MN-major A / B operand (0: K-major).
-__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t a_mn, uint32_t b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) | ((n >> 3) << 17) |
+// fmt: operand format, 1 = bf16, 0 = fp16 (both operands alike).
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t a_mn, uint32_t b_mn, uint32_t fmt = 1u) {
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (a_mn << 15) | (b_mn << 16) | ((n >> 3) << 17) |
            ((uint32_t)(BM >> 4) << 24);
 }
 
@@ -240,6 +247,62 @@ pack_kernel(const __grid_constant__ Batch batch, PackArgs a) {
         const int o = rho * 128 + img_chunk_offset(rho, c);
         *reinterpret_cast<uint4*>(out0 + o) = t0;
         *reinterpret_cast<uint4*>(out1 + o) = t1;
+        if (a.dst.planes == 3)
+            *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(w.scratch) +
+                                      img_row_offset(a.dst, 2, panel, (int64_t)rb * 128) + o) = half8(v, 1.f);
+    }
+}
+
+// fp16 plane of R for the single-pass fused feedback/update product.  R is scaled by the power of
+// two that brings its largest column norm to about 2^10 (no entry can then overflow fp16, and
+// typical entries stay far from the subnormal range); the inverse scale is left at `rscale_off`
+// for the epilogue.  cnorm holds the squared column norms of R (written by the Cholesky of the
+// right QR, or by ColNorm).  One CTA per (panel, 128-row block), 256 threads.
+struct PackHalfArgs {
+    int32_t rows, cols;
+    ImgRef dst;
+    int64_t cnorm_off, rscale_off;
+};
+
+__global__ void __launch_bounds__(256)
+pack_half_kernel(const __grid_constant__ Batch batch, PackHalfArgs a) {
+    const MatWork& w = batch.w[blockIdx.z];
+    if (*w.status & ST_FAILED) return;
+    __shared__ float red[8];
+    __shared__ float s_scale;
+    const float* cn = reinterpret_cast<const float*>(w.scratch + a.cnorm_off);
+    float mx = 0.f;
+    for (int j = threadIdx.x; j < a.cols; j += 256) mx = fmaxf(mx, cn[j]);
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (threadIdx.x % 32 == 0) red[threadIdx.x / 32] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+        int e = 0;
+        const float nrm = sqrtf(mx);
+        if (nrm > 0.f && nrm <= 3.0e38f) frexpf(nrm, &e);      // nrm = f * 2^e, 0.5 <= f < 1
+        const float scale = ldexpf(1.f, 10 - e);
+        s_scale = scale;
+        if (blockIdx.x == 0 && blockIdx.y == 0)
+            *reinterpret_cast<float*>(w.scratch + a.rscale_off) = ldexpf(1.f, e - 10);
+    }
+    __syncthreads();
+    const float scale = s_scale;
+    const int panel = blockIdx.x, rb = blockIdx.y;
+    unsigned char* out = reinterpret_cast<unsigned char*>(w.scratch) + img_row_offset(a.dst, 2, panel, (int64_t)rb * 128);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int q = threadIdx.x + 256 * e;
+        const int rho = q / 8, c = q % 8;
+        const int64_t gr = (int64_t)rb * 128 + rho, gk = (int64_t)panel * 64 + c * 8;
+        float v[8];
+        if (gr < a.rows && gk < a.cols) {
+            load8(w.R, gr * a.cols + gk, 0, v);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        }
+        *reinterpret_cast<uint4*>(out + rho * 128 + img_chunk_offset(rho, c)) = half8(v, scale);
     }
 }
 
@@ -247,9 +310,12 @@ pack_kernel(const __grid_constant__ Batch batch, PackArgs a) {
 // Tile bookkeeping shared by all roles of the GEMM kernel
 // ------------------------------------------------------------------------------------------
 struct TileCoord { int b, mt, nt, n0, bn, kb_end; bool active; };
+// Each role remembers the status word of the matrix it is working on (nothing changes it while
+// the kernel runs), so that only the first tile of a matrix pays for the global load.
+struct StatusCache { int b = -1; int st = 0; };
 
 template <int EPI>
-__device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmArgs& g, int t) {
+__device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmArgs& g, int t, StatusCache& sc) {
     TileCoord c;
     const int per = g.m_tiles * g.n_tiles;
     c.b = t / per;
@@ -260,7 +326,8 @@ __device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmA
     c.bn = min(g.BN, g.Ncols - c.n0);
     c.kb_end = g.k_blocks;
     if (g.tri) c.kb_end = min(g.k_blocks, (c.n0 + c.bn + BK - 1) / BK);
-    const int st = *batch.w[c.b].status;
+    if (c.b != sc.b) { sc.b = c.b; sc.st = *batch.w[c.b].status; }
+    const int st = sc.st;
     c.active = !(st & ST_FAILED);
     if (EPI != EPI_K5 && g.out.only_if_shifted && !(st & g.out.shift_bit)) c.active = false;
     if (g.lower_only && c.n0 > c.mt * BM + BM - 1) c.active = false;
@@ -314,20 +381,21 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);
     unsigned char* a_ring = smem;
-    unsigned char* n_ring = smem + A_SLOTS * A_SLOT_BYTES;
+    unsigned char* n_ring = smem + g.a_slots * g.a_slot_bytes;
     unsigned char* staging = n_ring + (size_t)g.n_slots * g.n_piece_bytes;
-    unsigned char* tail = staging + (EPI == EPI_K5 ? NE * STAGING_BYTES_PER_WARP : 0);
+    unsigned char* tail = staging + (EPI == EPI_K5 ? NE * g.epi_bufs * STAGING_BYTES_PER_WARP : 0);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
-    const uint32_t a_full0 = smem_u32(bars), a_empty0 = a_full0 + 8 * A_SLOTS;
-    const uint32_t n_full0 = a_empty0 + 8 * A_SLOTS, n_empty0 = n_full0 + 8 * MAX_N_SLOTS;
+    const uint32_t a_full0 = smem_u32(bars), a_empty0 = a_full0 + 8 * MAX_A_SLOTS;
+    const uint32_t n_full0 = a_empty0 + 8 * MAX_A_SLOTS, n_empty0 = n_full0 + 8 * MAX_N_SLOTS;
     const uint32_t tfull0 = n_empty0 + 8 * MAX_N_SLOTS, tempty0 = tfull0 + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * A_SLOTS + 2 * MAX_N_SLOTS + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_A_SLOTS + 2 * MAX_N_SLOTS + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    StatusCache scache;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < A_SLOTS; ++s) {
+        for (int s = 0; s < MAX_A_SLOTS; ++s) {
             mbar_init(a_full0 + 8 * s, A_BUF ? NUM_XF_WARPS : 1);
             mbar_init(a_empty0 + 8 * s, 1);
         }
@@ -350,89 +418,85 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t acc_stride = (uint32_t)(g.tmem_cols / g.acc_bufs);
 
-    const int a_terms = (g.passes == 3 || (EPI == EPI_K5 && g.passes2 == 3)) ? 2 : 1;
+    const int a_terms = g.a_slot_bytes / A_TERM_BYTES;
     const int n1_terms = g.passes == 3 ? 2 : 1;
+    const int plane = g.fp16 ? 2 : 0;
+    const uint32_t fmt = g.fp16 ? 0u : 1u;
     // N_IMG_MN piece geometry: [term][64-column group][ks rows of 128 bytes]
     const uint32_t group_stride = (uint32_t)g.ks * 128u;
     const uint32_t mn_term_stride = (uint32_t)((g.BN + 63) / 64) * group_stride;
 
     if (warp == 0) {
         // ---------------- producer ----------------
-        // Lane 0 arms the barrier of a slot and issues the one TMA load that fills it.  For the
-        // fused feedback/update pass the whole warp also asks for the next tile's M, G, X in L2,
-        // so that the epilogue's loads see L2 latency and need few bytes in flight.
-        {
+        // One thread feeds both rings.  It walks the schedule twice, with one cursor per ring, and
+        // serves whichever ring has a free slot, so a full N ring never holds back A tiles (and
+        // the other way round).  Every slot is filled by one tiled TMA load (two for the fused
+        // pass: R and Q pieces).
+        if (lane == 0) {
             int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
-            bool ok = true;
-            constexpr int GB = G_BF16 ? 2 : 4, XB = X_BF16 ? 2 : 4;
-            auto prefetch_k5 = [&](int t) {
-                if (t >= g.total_tiles) return;
-                const TileCoord c = decode_tile<EPI>(batch, g, t);
-                if (!c.active) return;
-                const MatWork& w = batch.w[c.b];
-                const int ncols = min(g.BN, g.Ncols - c.n0);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int64_t gi = (int64_t)c.mt * BM + lane + 32 * i;
-                    if (gi < g.Mrows) {
-                        const int64_t off = gi * g.ld + c.n0;
-                        const char* pm = reinterpret_cast<const char*>(w.M + off);
-                        const char* pg = reinterpret_cast<const char*>(w.G) + off * GB;
-                        const char* px = reinterpret_cast<const char*>(w.X) + off * XB;
-                        for (int o = 0; o < ncols * 4; o += 64) prefetch_l2(pm + o);
-                        for (int o = 0; o < ncols * GB; o += 64) prefetch_l2(pg + o);
-                        for (int o = 0; o < ncols * XB; o += 64) prefetch_l2(px + o);
-                    }
+            // cursor over (tile, depth block) for the A ring
+            int at = blockIdx.x, akb = 0; TileCoord ac{}; bool a_done = A_BUF;
+            // cursor over (tile, depth block, piece) for the N ring
+            int nt_ = blockIdx.x, nkb = 0, npc = 0; TileCoord nc{}; bool n_done = false;
+            auto a_seek = [&]() {           // make (at, akb) valid or finish
+                while (!a_done) {
+                    if (at >= g.total_tiles) { a_done = true; break; }
+                    if (akb == 0) ac = decode_tile<EPI>(batch, g, at, scache);
+                    if (ac.active && akb < ac.kb_end) break;
+                    at += gridDim.x; akb = 0;
                 }
             };
-            if (EPI == EPI_K5) prefetch_k5(blockIdx.x);
-            for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-                const TileCoord c = decode_tile<EPI>(batch, g, t);
-                if (EPI == EPI_K5) prefetch_k5(t + gridDim.x);
-                if (!c.active) continue;
-                for (int kb = 0; kb < c.kb_end && ok; ++kb) {
-                    if (!A_BUF) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(a_empty0 + 8 * as, aph ^ 1, abort_flag));
-                        if (!ok) break;
-                        if (lane == 0) {
-                            const uint32_t fb = a_full0 + 8 * as;
-                            const uint32_t dst = smem_u32(a_ring + as * A_SLOT_BYTES);
-                            mbar_arrive_expect_tx(fb, (uint32_t)a_terms * A_TERM_BYTES);
-                            if (AMODE == A_IMG_K) tma_load_box(dst, &g.map_a, c.mt * BM, kb, c.b, fb);
-                            else tma_load_box(dst, &g.map_a, kb * BK, c.mt * 2, c.b, fb);
-                        }
-                        if (++as == A_SLOTS) { as = 0; aph ^= 1; }
-                    }
+            auto n_pieces = [&](int kb) { return NMODE == N_IMG_MN ? mn_pieces(g, kb) : (nc.bn + 127) / 128; };
+            auto n_seek = [&]() {           // make (nt_, nkb, npc) valid or finish
+                while (!n_done) {
+                    if (nt_ >= g.total_tiles) { n_done = true; break; }
+                    if (nkb == 0 && npc == 0) nc = decode_tile<EPI>(batch, g, nt_, scache);
+                    if (!nc.active || nkb >= nc.kb_end) { nt_ += gridDim.x; nkb = 0; npc = 0; continue; }
+                    if (npc >= n_pieces(nkb)) { ++nkb; npc = 0; continue; }
+                    if (NMODE == N_IMG_K && !k_piece_active(g, nc, nkb, npc)) { ++npc; continue; }
+                    break;
+                }
+            };
+            a_seek();
+            n_seek();
+            long long idle_since = -1;
+            while (!a_done || !n_done) {
+                bool progress = false;
+                if (!a_done && mbar_try_wait(a_empty0 + 8 * as, aph ^ 1)) {
+                    const uint32_t fb = a_full0 + 8 * as;
+                    const uint32_t dst = smem_u32(a_ring + as * g.a_slot_bytes);
+                    mbar_arrive_expect_tx(fb, (uint32_t)a_terms * A_TERM_BYTES);
+                    if (AMODE == A_IMG_K) tma_load_box(dst, &g.map_a, ac.mt * BM, akb, plane, ac.b, fb);
+                    else tma_load_box(dst, &g.map_a, akb * BK, ac.mt * 2, plane, ac.b, fb);
+                    if (++as == g.a_slots) { as = 0; aph ^= 1; }
+                    ++akb;
+                    if (akb >= ac.kb_end) { at += gridDim.x; akb = 0; }
+                    a_seek();
+                    progress = true;
+                }
+                if (!n_done && mbar_try_wait(n_empty0 + 8 * ns, nph ^ 1)) {
+                    const uint32_t fb = n_full0 + 8 * ns;
+                    const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                    mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
                     if (NMODE == N_IMG_MN) {
-                        const int pieces = mn_pieces(g, kb);
-                        for (int sub = 0; sub < pieces && ok; ++sub) {
-                            ok = __all_sync(0xffffffffu, mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag));
-                            if (!ok) break;
-                            if (lane == 0) {
-                                const uint32_t fb = n_full0 + 8 * ns;
-                                mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
-                                tma_load_box(smem_u32(n_ring + (size_t)ns * g.n_piece_bytes), &g.map_n1,
-                                             kb * BK + sub * g.ks, c.n0 / 64, c.b, fb);
-                            }
-                            if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
-                        }
+                        tma_load_box(dst, &g.map_n1, nkb * BK + npc * g.ks, nc.n0 / 64, plane, nc.b, fb);
                     } else {
-                        const int chunks = (c.bn + 127) / 128;
-                        for (int ch = 0; ch < chunks && ok; ++ch) {
-                            if (!k_piece_active(g, c, kb, ch)) continue;
-                            ok = __all_sync(0xffffffffu, mbar_wait(n_empty0 + 8 * ns, nph ^ 1, abort_flag));
-                            if (!ok) break;
-                            if (lane == 0) {
-                                const uint32_t fb = n_full0 + 8 * ns;
-                                const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
-                                mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
-                                tma_load_box(dst, &g.map_n1, c.n0 + ch * 128, kb, c.b, fb);
-                                if (EPI == EPI_K5)
-                                    tma_load_box(dst + n1_terms * A_TERM_BYTES, &g.map_n2, c.n0 + ch * 128, kb, c.b, fb);
-                            }
-                            if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
-                        }
+                        tma_load_box(dst, &g.map_n1, nc.n0 + npc * 128, nkb, plane, nc.b, fb);
+                        if (EPI == EPI_K5)
+                            tma_load_box(dst + n1_terms * A_TERM_BYTES, &g.map_n2, nc.n0 + npc * 128, nkb, plane, nc.b, fb);
                     }
+                    if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
+                    ++npc;
+                    n_seek();
+                    progress = true;
+                }
+                if (progress) {
+                    idle_since = -1;
+                } else {
+                    if (*abort_flag) break;
+                    const long long now = clock64();
+                    if (idle_since < 0) idle_since = now;
+                    else if (now - idle_since > WAIT_LIMIT_CYCLES) { *abort_flag = 1; break; }
                 }
             }
         }
@@ -442,7 +506,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         int acc = 0; uint32_t acc_phase = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-            const TileCoord c = decode_tile<EPI>(batch, g, t);
+            const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
             if (!c.active) continue;
             if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -450,7 +514,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             for (int kb = 0; kb < c.kb_end && ok; ++kb) {
                 if (!mbar_wait(a_full0 + 8 * as, aph, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t sa = smem_u32(a_ring + as * A_SLOT_BYTES);
+                const uint32_t sa = smem_u32(a_ring + as * g.a_slot_bytes);
                 if (NMODE == N_IMG_MN) {
                     const int pieces = mn_pieces(g, kb);
                     for (int sub = 0; sub < pieces && ok; ++sub) {
@@ -469,7 +533,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                 const uint32_t accum = (kb > 0 || sub > 0 || j > 0) ? 1u : 0u;
                                 for (int cc = 0; cc < c.bn; cc += 256) {
                                     const uint32_t ncols = (uint32_t)min(256, c.bn - cc);
-                                    const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 1u);
+                                    const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 1u, fmt);
                                     const uint32_t nb = sn + (cc / 64) * group_stride + j * 2048;
                                     const uint64_t b0 = smem_desc(nb, group_stride, 1024);
                                     const uint64_t b1 = smem_desc(nb + mn_term_stride, group_stride, 1024);
@@ -495,7 +559,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                         if (lane == 0) {
                             const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
                             const uint32_t ncols = (uint32_t)min(128, c.bn - ch * 128);
-                            const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u);
+                            const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u, fmt);
                             for (int j = 0; j < nsl; ++j) {
                                 const uint64_t a0 = A_MN ? smem_desc(sa + j * 2048, 8192, 1024)
                                                          : smem_desc(sa + j * 32, 16, 1024);
@@ -531,7 +595,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 if (!ok) break;
                 if (lane == 0) umma_commit(a_empty0 + 8 * as);
                 __syncwarp();
-                if (++as == A_SLOTS) { as = 0; aph ^= 1; }
+                if (++as == g.a_slots) { as = 0; aph ^= 1; }
             }
             if (!ok) break;
             if (lane == 0) umma_commit(tfull0 + 8 * acc);
@@ -545,12 +609,12 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         const int quarter = warp % 4;                    // tensor-memory lanes 32*quarter .. +31
         if (EPI == EPI_STORE) {
             for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
                 if (!c.active) continue;
                 if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const MatWork& w = batch.w[c.b];
-                const int stw = *w.status;
+                const int stw = scache.st;
                 const Dest& d = (g.out.shift_bit && (stw & g.out.shift_bit)) ? g.out.shifted : g.out.normal;
                 const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16);
                 const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + lane;
@@ -590,6 +654,8 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                             const int o = img_chunk_offset((int)(gi & 7), ch0 + h);
                             *reinterpret_cast<uint4*>(r0 + o) = t0;
                             *reinterpret_cast<uint4*>(r1 + o) = t1;
+                            if (d.img.planes == 3)
+                                *reinterpret_cast<uint4*>(scr + img_row_offset(d.img, 2, panel, gi) + o) = half8(f, 1.f);
                         }
                     }
                     if (csq && cc < c.bn) {
@@ -627,17 +693,156 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             // along rows (8 lanes x 16 bytes per row).  The producer warp has already asked for the
             // tile's M, G, X in L2, so the loads of a slab return with L2 latency.
             const int half = (warp - 2) / 4;
+            auto next_tile = [&](int t) {
+                for (t += gridDim.x; t < g.total_tiles; t += gridDim.x)
+                    if (decode_tile<EPI>(batch, g, t, scache).active) return t;
+                return g.total_tiles;
+            };
+            // the slabs of this warp in order: (tile, 0), (tile, 1), (next tile, 0), ...
+            auto advance = [&](int& t, int& slab) {
+                if (++slab == 2) { slab = 0; t = next_tile(t); }
+            };
+            if constexpr (XG == 3) {
+                // bf16 G and X.  The 32 x 32 slabs of M, G, X come in by asynchronous copies
+                // (cp.async, no registers) into a per-warp buffer, one or two slabs ahead; each
+                // lane then updates its own row in place (accumulators stay in the layout tensor
+                // memory gives: one row per lane), and the buffer goes out along rows.
+                //   buffer: M 32 x 128 B | G 32 x 64 B | X 32 x 64 B, 16-byte chunks swizzled so that
+                //   both the row-per-lane and the 8-(or 4-)lanes-per-row accesses avoid bank conflicts
+                const int nbuf = g.epi_bufs;
+                unsigned char* bufs = staging + (size_t)(warp - 2) * nbuf * STAGING_BYTES_PER_WARP;
+                const int mrow = lane / 8, mch = lane % 8;      // M: 4 rows x 8 chunks per step
+                const int hrow = lane / 4, hch = lane % 4;      // G, X: 8 rows x 4 chunks per step
+                auto m_off = [](int r, int ch) { return r * 128 + ((ch ^ (r & 7)) << 4); };
+                auto h_off = [](int r, int ch) { return r * 64 + ((ch ^ ((r >> 1) & 3)) << 4); };
+                auto issue = [&](int t, int slab, unsigned char* buf) {
+                    const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+                    const MatWork& w = batch.w[c.b];
+                    const int64_t gj0 = (int64_t)c.n0 + half * 64 + slab * 32;
+                    const int64_t gi0 = (int64_t)c.mt * BM + quarter * 32;
+                    const uint32_t sb = smem_u32(buf);
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int r = it * 4 + mrow;
+                        const int64_t gi = gi0 + r, gj = gj0 + mch * 4;
+                        if (gi < g.Mrows && gj < g.Ncols) cp_async16(sb + m_off(r, mch), w.M + gi * g.ld + gj);
+                    }
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int r = it * 8 + hrow;
+                        const int64_t gi = gi0 + r, gj = gj0 + hch * 8;
+                        if (gi < g.Mrows && gj < g.Ncols) {
+                            const int64_t idx = gi * g.ld + gj;
+                            cp_async16(sb + 4096 + h_off(r, hch), reinterpret_cast<const __nv_bfloat16*>(w.G) + idx);
+                            cp_async16(sb + 6144 + h_off(r, hch), reinterpret_cast<const __nv_bfloat16*>(w.X) + idx);
+                        }
+                    }
+                    cp_async_commit();
+                };
+                auto process = [&](int t, int slab, unsigned char* buf) -> bool {
+                    const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+                    const MatWork& w = batch.w[c.b];
+                    const float efb = g.fp16 ? g.ef_b * *reinterpret_cast<const float*>(w.scratch + g.rscale_off) : g.ef_b;
+                    if (slab == 0) {
+                        if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) return false;
+                        tc_fence_after();
+                    }
+                    const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16) +
+                                           (uint32_t)(half * 64 + slab * 32);
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t va[16], vc[16];
+                        tmem_ld16(taddr + hh * 16, va);
+                        tmem_ld16(taddr + g.BN + hh * 16, vc);
+                        tmem_ld_wait();
+                        uint4 gq[2], xq[2];
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+                            gq[k] = *reinterpret_cast<const uint4*>(buf + 4096 + h_off(lane, hh * 2 + k));
+                            xq[k] = *reinterpret_cast<const uint4*>(buf + 6144 + h_off(lane, hh * 2 + k));
+                        }
+                        const uint32_t gw[8] = {gq[0].x, gq[0].y, gq[0].z, gq[0].w, gq[1].x, gq[1].y, gq[1].z, gq[1].w};
+                        const uint32_t xw[8] = {xq[0].x, xq[0].y, xq[0].z, xq[0].w, xq[1].x, xq[1].y, xq[1].z, xq[1].w};
+                        uint32_t xo[8];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            float4* mp = reinterpret_cast<float4*>(buf + m_off(lane, hh * 4 + k));
+                            const float4 mv = *mp;
+                            const float mvv[4] = {mv.x, mv.y, mv.z, mv.w};
+                            float mo[4], xf[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int i = 4 * k + e;
+                                const uint32_t gp = gw[i / 2], xp = xw[i / 2];
+                                const float gval = (i & 1) ? bf16hi_to_f32(gp) : bf16lo_to_f32(gp);
+                                const float xval = (i & 1) ? bf16hi_to_f32(xp) : bf16lo_to_f32(xp);
+                                const float bval = mvv[e] + gval;
+                                mo[e] = g.ef_a * bval - efb * __uint_as_float(va[i]);
+                                xf[e] = g.wc * xval - g.wd * __uint_as_float(vc[i]);
+                            }
+                            *mp = make_float4(mo[0], mo[1], mo[2], mo[3]);
+                            xo[2 * k] = pack_bf16x2(xf[0], xf[1]);
+                            xo[2 * k + 1] = pack_bf16x2(xf[2], xf[3]);
+                        }
+#pragma unroll
+                        for (int k = 0; k < 2; ++k)
+                            *reinterpret_cast<uint4*>(buf + 6144 + h_off(lane, hh * 2 + k)) =
+                                make_uint4(xo[4 * k], xo[4 * k + 1], xo[4 * k + 2], xo[4 * k + 3]);
+                    }
+                    if (slab == 1) {
+                        // the accumulators of this tile are in registers / shared memory now
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                        if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
+                    }
+                    __syncwarp();
+                    const int64_t gj0 = (int64_t)c.n0 + half * 64 + slab * 32;
+                    const int64_t gi0 = (int64_t)c.mt * BM + quarter * 32;
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int r = it * 4 + mrow;
+                        const int64_t gi = gi0 + r, gj = gj0 + mch * 4;
+                        if (gi < g.Mrows && gj < g.Ncols)
+                            *reinterpret_cast<float4*>(w.M + gi * g.ld + gj) = *reinterpret_cast<const float4*>(buf + m_off(r, mch));
+                    }
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int r = it * 8 + hrow;
+                        const int64_t gi = gi0 + r, gj = gj0 + hch * 8;
+                        if (gi < g.Mrows && gj < g.Ncols)
+                            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(w.X) + gi * g.ld + gj) =
+                                *reinterpret_cast<const uint4*>(buf + 6144 + h_off(r, hch));
+                    }
+                    __syncwarp();
+                    return true;
+                };
+                int t = next_tile(blockIdx.x - (int)gridDim.x), slab = 0, ib = 0;
+                if (t < g.total_tiles) issue(t, slab, bufs);
+                while (t < g.total_tiles) {
+                    int t2 = t, slab2 = slab;
+                    advance(t2, slab2);
+                    if (nbuf == 2) {
+                        if (t2 < g.total_tiles) issue(t2, slab2, bufs + (ib ^ 1) * STAGING_BYTES_PER_WARP);
+                        else cp_async_commit();
+                        cp_async_wait<1>();
+                    } else {
+                        cp_async_wait<0>();
+                    }
+                    __syncwarp();
+                    if (!process(t, slab, bufs + ib * STAGING_BYTES_PER_WARP)) break;
+                    if (nbuf == 2) ib ^= 1;
+                    else if (t2 < g.total_tiles) issue(t2, slab2, bufs);
+                    t = t2; slab = slab2;
+                }
+                cp_async_wait<0>();
+            } else {
             unsigned char* S1 = staging + (warp - 2) * STAGING_BYTES_PER_WARP;
             unsigned char* S2 = S1 + 4096;
             const int rl = lane / 8, cq = lane % 8;      // row within a step, 4-column group
 
-            auto next_tile = [&](int t) {
-                for (t += gridDim.x; t < g.total_tiles; t += gridDim.x)
-                    if (decode_tile<EPI>(batch, g, t).active) return t;
-                return g.total_tiles;
-            };
             auto fetch = [&](K5Pre<XG>& p, int t, int slab) {
-                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
                 const MatWork& w = batch.w[c.b];
                 const int64_t gj = (int64_t)c.n0 + half * 64 + slab * 32 + cq * 4;
 #pragma unroll
@@ -666,8 +871,9 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
 
             // one slab: accumulators -> staging -> row-wise update of M and X
             auto process = [&](const K5Pre<XG>& cur, int t, int slab) -> bool {
-                const TileCoord c = decode_tile<EPI>(batch, g, t);
+                const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
                 const MatWork& w = batch.w[c.b];
+                const float efb = g.fp16 ? g.ef_b * *reinterpret_cast<const float*>(w.scratch + g.rscale_off) : g.ef_b;
                 if (slab == 0) {
                     if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) return false;
                     tc_fence_after();
@@ -724,7 +930,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float bval = mv[e] + gv[e];
-                            mo[e] = g.ef_a * bval - g.ef_b * a1[e];
+                            mo[e] = g.ef_a * bval - efb * a1[e];
                             xo[e] = g.wc * xv[e] - g.wd * a2[e];
                         }
                         *reinterpret_cast<float4*>(w.M + idx) = make_float4(mo[0], mo[1], mo[2], mo[3]);
@@ -746,17 +952,13 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 }
                 return true;
             };
-            // the slabs of this warp in order: (tile, 0), (tile, 1), (next tile, 0), ...
-            auto advance = [&](int& t, int& slab) {
-                if (++slab == 2) { slab = 0; t = next_tile(t); }
-            };
-
             int t = next_tile(blockIdx.x - (int)gridDim.x), slab = 0;
             K5Pre<XG> pa;
             while (t < g.total_tiles) {
                 fetch(pa, t, slab);
                 if (!process(pa, t, slab)) break;
                 advance(t, slab);
+            }
             }
         }
     } else if (A_BUF) {
@@ -768,7 +970,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         bool ok = true;
         struct Raw { float4 m[2][2]; uint32_t gq[2][G_BF16 ? 4 : 8]; };
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-            const TileCoord c = decode_tile<EPI>(batch, g, t);
+            const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
             if (!c.active) continue;
             const MatWork& w = batch.w[c.b];
             const int64_t ld = g.ld;
@@ -840,7 +1042,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             // wait for the slot, store the tile, signal the MMA issuer
             auto store = [&](const uint4 (&t0)[2], const uint4 (&t1)[2]) -> bool {
                 if (!mbar_wait(a_empty0 + 8 * as, aph ^ 1, abort_flag)) return false;
-                unsigned char* sa = a_ring + as * A_SLOT_BYTES;
+                unsigned char* sa = a_ring + as * g.a_slot_bytes;
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     *reinterpret_cast<uint4*>(sa + dst_off[e]) = t0[e];
@@ -849,7 +1051,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(a_full0 + 8 * as);
-                if (++as == A_SLOTS) { as = 0; aph ^= 1; }
+                if (++as == g.a_slots) { as = 0; aph ^= 1; }
                 return true;
             };
             Raw r0, r1;
@@ -888,40 +1090,48 @@ struct TensorScratch {      // where the images of one matrix live inside its sc
     ImgRef linv;            // L^{-1} of the current Cholesky            (r x r)
     ImgRef qprev;           // Q_prev                                    (n x r)
     ImgRef w0, w1;          // Y = B Q_prev and the QR intermediates     (max(m,n) x r)
-    ImgRef p, r, q;         // P (m x r), R (n x r), Q (n x r)
+    ImgRef p, r, q;         // P (m x r), R (n x r), Q (n x r); three planes when the fused pass runs in fp16
     int64_t colsq;          // fp32 [4 * ceil(max(m,n)/128)][r] column-square partials
+    int64_t cnorm;          // fp32 [r] squared column norms of R
+    int64_t rscale;         // fp32 inverse of the scale of R's fp16 plane
 };
 
 inline bool tensor_engine_supports(int64_t m, int64_t n, int32_t r) {
     return r % 16 == 0 && n % 8 == 0 && m >= 1;
 }
 
-inline ImgRef make_img(int64_t off, int64_t rows, int64_t cols) {
+inline ImgRef make_img(int64_t off, int64_t rows, int64_t cols, int planes = 2) {
     ImgRef im;
     im.off = off;
     im.rows_pad = (int32_t)((rows + 127) / 128 * 128);
     im.panels = (int32_t)((cols + 63) / 64);
+    im.planes = planes;
+    im.pad = 0;
     return im;
 }
-inline int64_t img_bytes(int64_t rows, int64_t cols) {
-    return 2 * ((cols + 63) / 64) * ((rows + 127) / 128 * 128) * 128;
+inline int64_t img_bytes(int64_t rows, int64_t cols, int planes = 2) {
+    return planes * ((cols + 63) / 64) * ((rows + 127) / 128 * 128) * 128;
 }
-inline ImgRef no_img() { ImgRef im; im.off = -1; im.rows_pad = 0; im.panels = 0; return im; }
+inline ImgRef no_img() { ImgRef im; im.off = -1; im.rows_pad = 0; im.panels = 0; im.planes = 0; im.pad = 0; return im; }
 
 // The offsets of linv and colsq depend on r only, so that one Cholesky launch can serve
 // matrices of different shapes.
-inline size_t tensor_scratch_layout(int64_t m, int64_t n, int32_t r, size_t off, TensorScratch* ts) {
+// half_planes: P, R, Q carry the fp16 plane (fused pass in fp16).
+inline size_t tensor_scratch_layout(int64_t m, int64_t n, int32_t r, bool half_planes, size_t off, TensorScratch* ts) {
     const int64_t kmax = std::max(m, n);
     off = (off + 1023) / 1024 * 1024;
     auto take = [&](int64_t bytes) { int64_t o = (int64_t)off; off += (size_t)((bytes + 1023) / 1024 * 1024); return o; };
     ts->linv = make_img(take(img_bytes(r, r)), r, r);
     ts->colsq = take(4 * ((kmax + 127) / 128) * (int64_t)r * 4);
+    ts->cnorm = take((int64_t)r * 4);
+    ts->rscale = take(16);
+    const int pl = half_planes ? 3 : 2;
     ts->qprev = make_img(take(img_bytes(n, r)), n, r);
     ts->w0 = make_img(take(img_bytes(kmax, r)), kmax, r);
     ts->w1 = make_img(take(img_bytes(kmax, r)), kmax, r);
-    ts->p = make_img(take(img_bytes(m, r)), m, r);
-    ts->r = make_img(take(img_bytes(n, r)), n, r);
-    ts->q = make_img(take(img_bytes(n, r)), n, r);
+    ts->p = make_img(take(img_bytes(m, r, pl)), m, r, pl);
+    ts->r = make_img(take(img_bytes(n, r, pl)), n, r, pl);
+    ts->q = make_img(take(img_bytes(n, r, pl)), n, r, pl);
     return off;
 }
 // the work images are sized for max(m, n) rows; a product over `rows` rows sees this view
@@ -959,9 +1169,10 @@ inline void encode_img_map(CUtensorMap* map, const Batch& b, const ImgRef& img, 
     TensorMapEncodeFn enc = tensor_map_encoder();
     if (!enc) { engine_error() = 1; return; }
     const cuuint64_t term_bytes = (cuuint64_t)img.panels * img.rows_pad * 128;
-    cuuint64_t dims[5] = {64, (cuuint64_t)img.rows_pad, (cuuint64_t)img.panels, 2, (cuuint64_t)b.count};
+    cuuint64_t dims[5] = {64, (cuuint64_t)img.rows_pad, (cuuint64_t)img.panels, (cuuint64_t)img.planes,
+                          (cuuint64_t)b.count};
     cuuint64_t strides[4] = {128, (cuuint64_t)img.rows_pad * 128, term_bytes,
-                             b.count > 1 ? (cuuint64_t)b.scratch_stride : 2 * term_bytes};
+                             b.count > 1 ? (cuuint64_t)b.scratch_stride : img.planes * term_bytes};
     cuuint32_t box[5] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_panels, (cuuint32_t)box_terms, 1};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     void* base = b.w[0].scratch + img.off;
@@ -1008,6 +1219,14 @@ inline cudaError_t tensor_engine_set_attributes() {
     return cudaSuccess;
 }
 
+inline void launch_pack_half(const Batch& b, int64_t rows, int64_t cols, const TensorScratch& ts, cudaStream_t st) {
+    tc::PackHalfArgs a{};
+    a.rows = (int32_t)rows; a.cols = (int32_t)cols; a.dst = ts.r; a.cnorm_off = ts.cnorm; a.rscale_off = ts.rscale;
+    dim3 grid((unsigned)ts.r.panels, (unsigned)(ts.r.rows_pad / 128), (unsigned)b.count);
+    prof::Scope scope(prof::S_PACK, st);
+    tc::pack_half_kernel<<<grid, 256, 0, st>>>(b, a);
+}
+
 inline void launch_pack(const Batch& b, Sel src, int64_t rows, int64_t cols, ImgRef dst, cudaStream_t st) {
     tc::PackArgs a{};
     a.src = src; a.rows = (int32_t)rows; a.cols = (int32_t)cols; a.dst = dst;
@@ -1023,8 +1242,19 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     g.n_tiles = (g.Ncols + g.BN - 1) / g.BN;
     g.k_blocks = (g.Kdim + tc::BK - 1) / tc::BK;
     g.total_tiles = b.count * g.m_tiles * g.n_tiles;
+    if (g.fp16) { g.passes = 1; g.passes2 = 1; }
     const int n1_terms = g.passes == 3 ? 2 : 1, n2_terms = g.passes2 == 3 ? 2 : 1;
     const int bn64 = (g.BN + 63) / 64 * 64;
+    const int a_terms = (tc::a_is_buf(AMODE) || g.passes == 3 || (EPI == tc::EPI_K5 && g.passes2 == 3)) ? 2 : 1;
+    g.a_slot_bytes = a_terms * tc::A_TERM_BYTES;
+    g.a_slots = tc::A_RING_BYTES / g.a_slot_bytes;
+    g.epi_bufs = 1;
+    if (EPI == tc::EPI_K5) {
+        // the fused pass needs little MMA time per tile: two slots per ring, and (bf16 G and X,
+        // single-pass operands) a second epilogue buffer per warp instead
+        g.a_slots = (a_terms == 1) ? 4 : 2;
+        if (XG == 3 && a_terms == 1) g.epi_bufs = 1;
+    }
     if (NMODE == tc::N_IMG_MN) {
         g.ks = bn64 <= 128 ? 64 : (bn64 <= 256 ? 32 : 16);
         g.n_piece_bytes = n1_terms * (bn64 / 64) * g.ks * 128;
@@ -1037,12 +1267,11 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     int cols = 32;
     while (cols < g.acc_bufs * accw) cols *= 2;
     g.tmem_cols = cols;
-    const size_t fixed = (size_t)tc::A_SLOTS * tc::A_SLOT_BYTES +
-                         (EPI == tc::EPI_K5 ? tc::epi_warps(EPI) * tc::STAGING_BYTES_PER_WARP : 0) + 256 + 1024;
+    const size_t fixed = (size_t)g.a_slots * g.a_slot_bytes +
+                         (EPI == tc::EPI_K5 ? tc::epi_warps(EPI) * g.epi_bufs * tc::STAGING_BYTES_PER_WARP : 0) + 256 + 1024;
     g.n_slots = (int)std::min<size_t>(tc::MAX_N_SLOTS, (tc::SMEM_LIMIT - fixed) / (size_t)g.n_piece_bytes);
     // more than half of an SM's shared memory: one CTA per SM, whatever its tensor-memory share
     const size_t smem = std::max<size_t>(fixed + (size_t)g.n_slots * g.n_piece_bytes, 120 * 1024);
-    const int a_terms = (g.passes == 3 || (EPI == tc::EPI_K5 && g.passes2 == 3)) ? 2 : 1;
     if (AMODE == tc::A_IMG_K) encode_img_map(&g.map_a, b, g.a, 128, 1, a_terms);
     else if (AMODE == tc::A_IMG_MN) encode_img_map(&g.map_a, b, g.a, 64, 2, a_terms);
     if (NMODE == tc::N_IMG_MN) encode_img_map(&g.map_n1, b, g.n1, g.ks, bn64 / 64, n1_terms);
@@ -1112,9 +1341,13 @@ inline void tensor_apply(int r, int passes, const Batch& b, const TensorScratch&
 }
 
 // M <- a (M + G) - b P R^T ;  X <- c X - d P Q^T                  (Alg. 1 lines 5-7)
-inline void tensor_k5(int64_t m, int64_t n, int r, int g_bf16, int x_bf16, int passes_m, int passes_x, float ef_a,
-                      float ef_b, float wc, float wd, const Batch& b, const TensorScratch& ts, cudaStream_t st) {
+// fp16 = 1: both products run as one fp16 pass from the fp16 planes of P, R, Q (R's plane must
+// have been written by launch_pack_half).
+inline void tensor_k5(int64_t m, int64_t n, int r, int g_bf16, int x_bf16, int passes_m, int passes_x, int fp16,
+                      float ef_a, float ef_b, float wc, float wd, const Batch& b, const TensorScratch& ts,
+                      cudaStream_t st) {
     tc::GemmArgs g{};
+    g.fp16 = fp16; g.rscale_off = ts.rscale;
     g.Mrows = (int32_t)m; g.Ncols = (int32_t)n; g.Kdim = r; g.BN = 128;
     g.passes = passes_m; g.passes2 = passes_x; g.ld = n;
     g.a = ts.p; g.n1 = ts.r; g.n2 = ts.q;

@@ -34,8 +34,9 @@ def make_problem(m, n, r, xdt, gdt, seed, m_scale=0.3):
 
 
 def one_step_compare(spec, X, M, G, Q, *, mode, engine, mu=0.95, eta=0.01, wd=0.0, ef=None, scale=None,
-                     tol=TOL_STEP):
-    gm = GpuMatrix(spec, X, M, Q, mu=mu, eta=eta, wd=wd, mode=mode, engine=engine, ef=ef, scale=scale)
+                     tol=TOL_STEP, passes=None):
+    gm = GpuMatrix(spec, X, M, Q, mu=mu, eta=eta, wd=wd, mode=mode, engine=engine, ef=ef, scale=scale,
+                   passes=passes)
     gm.step(G)
     assert gm.status() & ~(od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT) == 0
     kw = dict(ef=ef) if ef is not None else dict(mu=mu)
@@ -121,6 +122,18 @@ def test_one_step_tensor_shapes(shape, mode, dt):
     m, n, r = shape
     spec, X, M, G, Q = make_problem(m, n, r, dt[0], dt[1], seed=m * 7 + n)
     one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_TENSOR)
+
+
+@pytest.mark.parametrize("shape", [(384, 640, 64), (1000, 264, 128), (136, 2056, 32), (640, 384, 272)])
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("m_scale", [0.3, 3e-4, 300.0])
+def test_one_step_fused_pass_in_fp16(shape, mode, m_scale):
+    # the error-feedback and weight-update products as one fp16 pass (R scaled by a power of two):
+    # same tolerances, also when the buffer is far from unit scale
+    m, n, r = shape
+    spec, X, M, G, Q = make_problem(m, n, r, BF16, BF16, seed=m * 3 + n, m_scale=m_scale)
+    G = (G.float() * (m_scale / 0.3)).to(BF16)
+    one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_TENSOR, passes={2: 1, 3: 1})
 
 
 @pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
@@ -245,12 +258,14 @@ def test_state_is_only_m_and_q(engine):
 
 # ------------------------------------------------------------------ cfg1: 4096 x 4096, r = 256, bf16
 @pytest.mark.parametrize("mode", MODES)
-def test_cfg1_first_steps(mode):
+@pytest.mark.parametrize("fused", ["bf16x3", "fp16"])
+def test_cfg1_first_steps(mode, fused):
     w = wl.workload("cfg1")
     spec = w.matrices[0]
     X, M, Q = wl.initial_state(spec, 0, 0)
     basis = wl.grad_basis(w, spec, 0, 0)
-    gm = GpuMatrix(spec, X, M, Q, mu=w.mu, eta=w.eta, wd=w.wd, mode=mode)
+    gm = GpuMatrix(spec, X, M, Q, mu=w.mu, eta=w.eta, wd=w.wd, mode=mode,
+                   passes={2: 1, 3: 1} if fused == "fp16" else {2: 3, 3: 1})
     Xo, Mo, Qo = f64(X), f64(M), f64(Q)
     for t in range(3):
         G = wl.gradient(w, spec, 0, 0, t, basis)
