@@ -5,9 +5,9 @@
 
 namespace od {
 
-constexpr int CH_THREADS = 1024;
+constexpr int CH_THREADS = 512;               // two CTAs (two matrices) share an SM
 constexpr int CH_NB = 32;                      // panel / diagonal block width
-constexpr int CH_GROUPS = CH_THREADS / 256;    // 4 groups of 256 threads run 64x64 tile products
+constexpr int CH_GROUPS = CH_THREADS / 256;    // groups of 256 threads run 64x64 tile products
 constexpr int CH_DIAG_WARPS = 16;              // diagonal blocks inverted concurrently
 constexpr size_t CH_SMEM_BYTES =
     (size_t)CH_GROUPS * 2 * 16 * 65 * 4 + (size_t)CH_DIAG_WARPS * 32 * 33 * 4 + 64;
@@ -84,7 +84,7 @@ struct CholArgs {
 // Factor Gram = L L^T (blocked, right-looking) and overwrite `work` with L^{-1}.
 // Pass 1 retries once with a diagonal shift when the factorisation breaks down or looks
 // ill-conditioned, and records that in the status word so that a third QR pass is run.
-__global__ void __launch_bounds__(CH_THREADS, 1)
+__global__ void __launch_bounds__(CH_THREADS, 2)
 chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* gemm_smem = reinterpret_cast<float*>(smem_raw);
@@ -132,7 +132,7 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         if (lane == 0) red[warp] = t;
         __syncthreads();
         if (warp == 0) {
-            t = red[lane];
+            t = lane < CH_THREADS / 32 ? red[lane] : 0.f;
             for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
             if (lane == 0) s_trace = t;
         }
