@@ -9,7 +9,9 @@ factor, right QR or ColNorm, error feedback and weight update) over every weight
 8B Llama-style model (224 matrices, r = 512) with synthetic gradients.  `value` is parameter
 elements per second with everything resident in HBM; `e2e` is the same with the gradients coming
 from pinned host memory and the updated weights going back, copies inside the timed region.
-For N > 1 (torchrun) every rank steps its own replica of the model: no collective on the path.
+For N > 1 (torchrun) every rank steps its own replica of the model (--scaling weak, the default)
+or its share of the model's matrices (--scaling strong, whole matrices split by cost); either way
+there is no collective on the data path, and the step time is the maximum over the ranks.
 """
 from __future__ import annotations
 
@@ -28,6 +30,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2605_16341_b200 import sharding  # noqa: E402
 from paper_2605_16341_b200 import workloads as wl  # noqa: E402
 
 METRIC = "orthdion_step_param_elements_per_s"
@@ -212,6 +215,11 @@ def run_ours(args):
     w = wl.workload(args.workload, layers=args.layers, r=args.rank)
     mode = od.MODE_ORTH if args.mode == "orth" else od.MODE_COLNORM
     seed = 1000 + rank
+    all_matrices = w.matrices
+    if args.scaling == "strong" and world > 1:
+        mine = sharding.partition_matrices([(s.m, s.n, s.r) for s in all_matrices], world)[rank]
+        w = wl.Workload(w.name, tuple(all_matrices[i] for i in mine), w.grad, w.mu, w.eta, w.wd, w.grad_params)
+        seed = 1000
     hs, Xs, Ms, Qs, Gsets = [], [], [], [], [[] for _ in range(args.grad_sets)]
     plan_cache = {}
     for i, spec in enumerate(w.matrices):
@@ -270,18 +278,15 @@ def run_ours(args):
     launches = od.orthdion_launch_count() - l0
     stage_ms = od.orthdion_profile_end() if profile_on else {}
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    ms_total = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = sharding.max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     ms_step = ms_total / args.steps
     flags = od.orthdion_last_status(hs, ws, stream)
     failed = sum(1 for f in flags if f & (od.STATUS_RANK_DEFICIENT | od.STATUS_NONFINITE | od.STATUS_WAIT_LIMIT))
     shifted = sum(1 for f in flags if f & (od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT))
 
-    elements = w.numel
-    value = elements * world / (ms_step * 1e-3)
+    # elements stepped by the whole job: N replicas (weak) or the one model split N ways (strong)
+    elements = w.numel * world if args.scaling == "weak" else sum(s.numel for s in all_matrices)
+    value = elements / (ms_step * 1e-3)
 
     # ---- end to end: gradients from pinned host memory, updated weights back to the host ----
     e2e = None
@@ -347,10 +352,10 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": args.scaling,
         "vs_baseline": None, "dtype": "bf16-split products, f32 accumulate and state",
         "data": "synthetic",
-        "config": {"workload": f"{w.name}: {len(w.matrices)} matrices, {elements / 1e6:.1f}M elements, r={w.matrices[0].r}, "
+        "config": {"workload": f"{w.name}: {len(w.matrices)} matrices per rank, {elements / 1e6:.1f}M elements in the job, r={w.matrices[0].r}, "
                                f"bf16 X/G, fp32 M, mode {args.mode}",
                    "engine": args.engine, "l2": "inputs (tens of GB per step) far exceed the 126 MB L2",
                    "grad_sets": args.grad_sets, "replicas": world,
@@ -405,13 +410,14 @@ def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):
         one()
     ev1.record(stream)
     torch.cuda.synchronize()
-    ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     ms_step = ms / steps
-    return {"value": w.numel * world / (ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    job_elements = float(w.numel * world)
+    if args.scaling == "strong" and dist is not None:
+        t = torch.tensor([float(w.numel)], device=dev, dtype=torch.float64)
+        dist.all_reduce(t)
+        job_elements = float(t.item())
+    return {"value": job_elements / (ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms_step, "steps": steps}
 
 
@@ -425,6 +431,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="truncate the grouped models (experiments)")
     ap.add_argument("--rank", type=int, default=None, help="override r (cfg2 sweep)")
     ap.add_argument("--mode", default="orth", choices=["orth", "colnorm"])
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: one model replica per rank (weak) or the model's matrices split over ranks (strong)")
     ap.add_argument("--engine", default="tensor", choices=["tensor", "simt"])
     ap.add_argument("--passes", default=None,
                     help="bf16 split passes of the four product groups, e.g. 3,3,3,1 (0 keeps the default)")
