@@ -35,7 +35,7 @@ constexpr int A_RING_BYTES = 4 * A_TERM_BYTES;   // two slots of two terms, or f
 constexpr int MAX_A_SLOTS = 4;
 constexpr int MAX_N_SLOTS = 6;
 constexpr int NUM_XF_WARPS = 16;             // transform warps of the kernels that form B = M + G
-constexpr int STAGING_BYTES_PER_WARP = 8192; // K5 epilogue: two 32 x 32 fp32 blocks per warp
+constexpr int STAGING_BYTES_PER_WARP = 8192; // epilogue staging: one 32 x 64 fp32 block (or M, G, X slabs) per warp
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 
@@ -383,7 +383,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     unsigned char* a_ring = smem;
     unsigned char* n_ring = smem + g.a_slots * g.a_slot_bytes;
     unsigned char* staging = n_ring + (size_t)g.n_slots * g.n_piece_bytes;
-    unsigned char* tail = staging + (EPI == EPI_K5 ? NE * g.epi_bufs * STAGING_BYTES_PER_WARP : 0);
+    unsigned char* tail = staging + ((EPI == EPI_K5 || !A_BUF) ? NE * g.epi_bufs * STAGING_BYTES_PER_WARP : 0);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
     const uint32_t a_full0 = smem_u32(bars), a_empty0 = a_full0 + 8 * MAX_A_SLOTS;
     const uint32_t n_full0 = a_empty0 + 8 * MAX_A_SLOTS, n_empty0 = n_full0 + 8 * MAX_N_SLOTS;
@@ -617,12 +617,15 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 const int stw = scache.st;
                 const Dest& d = (g.out.shift_bit && (stw & g.out.shift_bit)) ? g.out.shifted : g.out.normal;
                 const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16);
-                const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + lane;
                 float* C = d.has_f32 ? pick(w, d.f32) : nullptr;
                 unsigned char* scr = reinterpret_cast<unsigned char*>(w.scratch);
                 const bool to_img = d.img.off >= 0;
                 float* csq = d.colsq ? reinterpret_cast<float*>(w.scratch + g.colsq_off) +
                                            (int64_t)(c.mt * 4 + quarter) * g.Ncols : nullptr;
+                if constexpr (A_BUF) {
+                // One wide tile per long main loop: the epilogue is a small share of the time, so
+                // it stores row per lane, 16 columns at a time, straight from the registers.
+                const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + lane;
                 const int bn64 = to_img ? (c.bn + 63) / 64 * 64 : c.bn;
                 for (int cc = 0; cc < bn64; cc += 16) {
                     uint32_t v[16];
@@ -680,6 +683,95 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                         const int col = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
                         if (!(lane & 1)) csq[gj + col] = s[0];
                     }
+                }
+                } else {
+                // 64 columns at a time: this warp's 32 x 64 block goes through an 8 KB staging
+                // buffer so that global stores run along rows.  A plane's block is 32 image rows of
+                // 128 bytes, byte for byte what the image holds, so it leaves as one 4 KB run.
+                unsigned char* stg = staging + (warp - 2) * STAGING_BYTES_PER_WARP;
+                const int64_t gi0 = (int64_t)c.mt * BM + quarter * 32;
+                const int groups = (c.bn + 63) / 64;
+                for (int cg = 0; cg < groups; ++cg) {
+                    const int valid = min(64, c.bn - cg * 64);          // multiple of 16
+                    const int gj0 = c.n0 + cg * 64;
+                    float f[64];
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t v[16];
+                        if (q4 * 16 < valid) {
+                            tmem_ld16(taddr + cg * 64 + q4 * 16, v);
+                            tmem_ld_wait();
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] = 0u;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) f[q4 * 16 + i] = __uint_as_float(v[i]);
+                        if (csq && q4 * 16 < valid) {
+                            // column sums of squares over the 32 rows of this warp: fold 16 values
+                            // over the lane bits 4..1, then add the two lanes that hold the same column
+                            float s[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) { const float x = __uint_as_float(v[i]); s[i] = x * x; }
+#pragma unroll
+                            for (int half = 8, bit = 16; half >= 1; half >>= 1, bit >>= 1) {
+                                const bool up = (lane & bit) != 0;
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    if (i < half) {
+                                        const float send = up ? s[i] : s[i + half];
+                                        const float keep = up ? s[i + half] : s[i];
+                                        s[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+                                    }
+                                }
+                            }
+                            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
+                            const int col = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+                            if (!(lane & 1)) csq[gj0 + q4 * 16 + col] = s[0];
+                        }
+                    }
+                    if (C) {
+                        // fp32 block: 32 rows x 256 bytes, 16-byte chunks swizzled by (row & 7)
+#pragma unroll
+                        for (int ch = 0; ch < 16; ++ch)
+                            *reinterpret_cast<float4*>(stg + lane * 256 + ((ch ^ (lane & 7)) << 4)) =
+                                make_float4(f[4 * ch], f[4 * ch + 1], f[4 * ch + 2], f[4 * ch + 3]);
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < 16; ++it) {
+                            const int r = it * 2 + lane / 16, ch = lane % 16;
+                            const float4 x = *reinterpret_cast<const float4*>(stg + r * 256 + ((ch ^ (r & 7)) << 4));
+                            if (gi0 + r < g.Mrows && ch * 4 < valid)
+                                *reinterpret_cast<float4*>(C + (gi0 + r) * g.out.ld + gj0 + ch * 4) = x;
+                        }
+                        __syncwarp();
+                    }
+                    if (to_img) {
+                        const int panel = gj0 / 64;
+                        for (int plane = 0; plane < d.img.planes; ++plane) {
+#pragma unroll
+                            for (int ch = 0; ch < 8; ++ch) {
+                                const float fv[8] = {f[8 * ch], f[8 * ch + 1], f[8 * ch + 2], f[8 * ch + 3],
+                                                     f[8 * ch + 4], f[8 * ch + 5], f[8 * ch + 6], f[8 * ch + 7]};
+                                uint4 t0, t1, out;
+                                if (plane == 2) {
+                                    out = half8(fv, 1.f);
+                                } else {
+                                    split8(fv, t0, t1);
+                                    out = plane == 0 ? t0 : t1;
+                                }
+                                *reinterpret_cast<uint4*>(stg + lane * 128 + img_chunk_offset(lane, ch)) = out;
+                            }
+                            __syncwarp();
+                            unsigned char* dst = scr + img_row_offset(d.img, plane, panel, gi0);
+#pragma unroll
+                            for (int it = 0; it < 8; ++it)
+                                *reinterpret_cast<uint4*>(dst + it * 512 + lane * 16) =
+                                    *reinterpret_cast<const uint4*>(stg + it * 512 + lane * 16);
+                            __syncwarp();
+                        }
+                    }
+                }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -1268,7 +1360,8 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     while (cols < g.acc_bufs * accw) cols *= 2;
     g.tmem_cols = cols;
     const size_t fixed = (size_t)g.a_slots * g.a_slot_bytes +
-                         (EPI == tc::EPI_K5 ? tc::epi_warps(EPI) * g.epi_bufs * tc::STAGING_BYTES_PER_WARP : 0) + 256 + 1024;
+                         (tc::a_is_buf(AMODE) ? 0 : (size_t)tc::epi_warps(EPI) * g.epi_bufs * tc::STAGING_BYTES_PER_WARP) +
+                         256 + 1024;
     g.n_slots = (int)std::min<size_t>(tc::MAX_N_SLOTS, (tc::SMEM_LIMIT - fixed) / (size_t)g.n_piece_bytes);
     // more than half of an SM's shared memory: one CTA per SM, whatever its tensor-memory share
     const size_t smem = std::max<size_t>(fixed + (size_t)g.n_slots * g.n_piece_bytes, 120 * 1024);
