@@ -1,0 +1,450 @@
+// r x r factor kernel of the tensor-core engine: blocked Cholesky of the Gram matrix and the
+// explicit inverse of its lower factor, one CTA (256 threads) per matrix, two CTAs per SM.
+//
+// Everything of cubic cost is a list of independent 64 x 64 tile products run on the warp-level
+// tensor-core path (mma.sync m16n8k16, bf16 operands, fp32 accumulation).  Operands are split into
+// two bf16 terms when they are staged in shared memory, and every 16 x 8 fragment is the sum of
+// three products (hi*hi + hi*lo + lo*hi): about 2^-16 relative accuracy per product.  (The first
+// QR pass only has to tame the condition number; in the second pass the factor is close to the
+// identity, so its off-diagonal products are small and their absolute error far below 1e-6.)
+// The global loads of the next 32-deep chunk (of this tile or of the next one) are issued before
+// the current chunk is multiplied, so the L2 latency hides behind the work.
+//
+// Right-looking Cholesky with 32-wide panels:
+//   diagonal block   one warp, rows in registers, pivots and columns passed by shuffles; its
+//                    inverse (needed at the end anyway) replaces it in place right away
+//   panel            rows below  <-  rows below * inv(L_kk)^T          (tile products, depth 32)
+//   trailing update  W22 -= L21 L21^T, lower tiles only                (tile products, depth 32)
+// then the inverse of the factor by combining diagonal blocks pairwise (32, 64, 128, ...):
+//   inv [[A, 0], [B, C]] = [[Ai, 0], [-Ci B Ai, Ci]]                   (tile products)
+#pragma once
+#include "common.cuh"
+#include "factor_kernels.cuh"
+
+namespace od {
+
+constexpr int CT_THREADS = 256;
+constexpr int CT_NB = 32;
+constexpr int CT_KC = 32;             // depth of one staged chunk
+constexpr int CT_LDK = 40;            // staged rows: 32 bf16 + 8 of padding (conflict-free fragment loads)
+constexpr int CT_MAX_TASKS = 160;
+
+// C(i,j) = beta*C(i,j) + alpha * sum_{k in [kbeg,kend)} A(i,k) B(k,j), i < Mt <= 64, j < Nt <= 64.
+// A(i,k) = A[i*a_rs + k];  B(k,j) = B[k*b_rs + j*b_cs] with b_rs == 1 (k contiguous) or b_cs == 1.
+struct TcTask {
+    float* C; const float* A; const float* B;
+    int32_t c_rs, c_cs, a_rs, b_rs, b_cs;
+    int32_t Mt, Nt, kbeg, kend, lower_only, rg0, cg0;
+    float alpha, beta;
+};
+
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// All 256 threads.  Warp w owns rows 16*(w % 4).., columns 32*(w / 4).. of the tile.
+__device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* stage) {
+    if (ntasks <= 0) return;
+    __nv_bfloat16* Ah = stage;
+    __nv_bfloat16* Al = Ah + 64 * CT_LDK;
+    __nv_bfloat16* Bh = Al + 64 * CT_LDK;
+    __nv_bfloat16* Bl = Bh + 64 * CT_LDK;
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int gq = lane / 4, tq = lane % 4;
+    const int row0 = (warp % 4) * 16, col0 = (warp / 4) * 32;
+    // Staging: a thread handles pairs of adjacent depth indices (one float2 load, one packed
+    // bf16x2 store per term): A rows a_ii + 16 e at depth a_kk, a_kk + 1; B likewise when depth is
+    // contiguous in memory, else single elements (jj = tid % 64, depth tid / 64 + 4 e).
+    const int a_kk = (tid % 16) * 2, a_ii = tid / 16;
+    float2 ra[4];
+    float rb[8];
+    auto load = [&](int task, int k0) {
+        const TcTask& t = tasks[task];
+        // kbeg, kend, a_rs are even and rows 8-byte aligned in all task lists of this file
+        const float* Ap = t.A + (a_ii * t.a_rs + k0 + a_kk);
+        const bool ak = k0 + a_kk < t.kend;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            ra[e] = (ak && a_ii + 16 * e < t.Mt) ? *reinterpret_cast<const float2*>(Ap + e * 16 * t.a_rs) : make_float2(0.f, 0.f);
+        if (t.b_rs == 1) {
+            const float* Bp = t.B + (k0 + a_kk + a_ii * t.b_cs);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 v = (ak && a_ii + 16 * e < t.Nt) ? *reinterpret_cast<const float2*>(Bp + e * 16 * t.b_cs)
+                                                              : make_float2(0.f, 0.f);
+                rb[2 * e] = v.x; rb[2 * e + 1] = v.y;
+            }
+        } else {
+            const int jj = tid % 64, kk = tid / 64;
+            const float* Bp = t.B + ((k0 + kk) * t.b_rs + jj);
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                rb[e] = (jj < t.Nt && k0 + kk + 4 * e < t.kend) ? Bp[e * 4 * t.b_rs] : 0.f;
+        }
+    };
+    int ti = 0, k0 = tasks[0].kbeg;
+    load(ti, k0);
+    float acc[4][4] = {};
+    while (true) {
+        {
+            const bool b_kfast = tasks[ti].b_rs == 1;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t hi = pack_bf16x2(ra[e].x, ra[e].y);
+                const uint32_t lo = pack_bf16x2(ra[e].x - bf16lo_to_f32(hi), ra[e].y - bf16hi_to_f32(hi));
+                const int oa = (a_ii + 16 * e) * CT_LDK + a_kk;
+                *reinterpret_cast<uint32_t*>(Ah + oa) = hi;
+                *reinterpret_cast<uint32_t*>(Al + oa) = lo;
+                if (b_kfast) {
+                    const uint32_t bhi = pack_bf16x2(rb[2 * e], rb[2 * e + 1]);
+                    const uint32_t blo = pack_bf16x2(rb[2 * e] - bf16lo_to_f32(bhi), rb[2 * e + 1] - bf16hi_to_f32(bhi));
+                    *reinterpret_cast<uint32_t*>(Bh + oa) = bhi;
+                    *reinterpret_cast<uint32_t*>(Bl + oa) = blo;
+                }
+            }
+            if (!b_kfast) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const __nv_bfloat16 bh = __float2bfloat16_rn(rb[e]);
+                    const int ob = (tid % 64) * CT_LDK + tid / 64 + 4 * e;
+                    Bh[ob] = bh;
+                    Bl[ob] = __float2bfloat16_rn(rb[e] - __bfloat162float(bh));
+                }
+            }
+        }
+        __syncthreads();
+        const bool last_chunk = k0 + CT_KC >= tasks[ti].kend;
+        int nti = ti, nk0 = k0 + CT_KC;
+        if (last_chunk) { nti = ti + 1; nk0 = nti < ntasks ? tasks[nti].kbeg : 0; }
+        const bool has_next = nti < ntasks;
+        if (has_next) load(nti, nk0);
+#pragma unroll
+        for (int ks = 0; ks < CT_KC; ks += 16) {
+            uint32_t ah[4], al[4];
+            const int o0 = (row0 + gq) * CT_LDK + ks + tq * 2, o1 = o0 + 8 * CT_LDK;
+            ah[0] = *reinterpret_cast<const uint32_t*>(Ah + o0);     al[0] = *reinterpret_cast<const uint32_t*>(Al + o0);
+            ah[1] = *reinterpret_cast<const uint32_t*>(Ah + o1);     al[1] = *reinterpret_cast<const uint32_t*>(Al + o1);
+            ah[2] = *reinterpret_cast<const uint32_t*>(Ah + o0 + 8); al[2] = *reinterpret_cast<const uint32_t*>(Al + o0 + 8);
+            ah[3] = *reinterpret_cast<const uint32_t*>(Ah + o1 + 8); al[3] = *reinterpret_cast<const uint32_t*>(Al + o1 + 8);
+#pragma unroll
+            for (int nf = 0; nf < 4; ++nf) {
+                const int o = (col0 + nf * 8 + gq) * CT_LDK + ks + tq * 2;
+                uint32_t bh[2], bl[2];
+                bh[0] = *reinterpret_cast<const uint32_t*>(Bh + o);     bl[0] = *reinterpret_cast<const uint32_t*>(Bl + o);
+                bh[1] = *reinterpret_cast<const uint32_t*>(Bh + o + 8); bl[1] = *reinterpret_cast<const uint32_t*>(Bl + o + 8);
+                mma_bf16_16x8x16(acc[nf], ah, bh);
+                mma_bf16_16x8x16(acc[nf], ah, bl);
+                mma_bf16_16x8x16(acc[nf], al, bh);
+            }
+        }
+        __syncthreads();
+        if (last_chunk) {
+            const TcTask& t = tasks[ti];
+            // all reads of C first, then all writes: a load behind a store that may alias it would
+            // wait for that store, and the sixteen round trips would line up one after the other
+            if (t.c_cs == 1) {
+                // rows of C are contiguous: the two columns of a fragment row go as one float2
+                float2 cv2[4][2];
+                bool v0[4][2], v1[4][2];
+#pragma unroll
+                for (int nf = 0; nf < 4; ++nf)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int i = row0 + gq + h * 8, j = col0 + nf * 8 + tq * 2;
+                        v0[nf][h] = i < t.Mt && j < t.Nt && !(t.lower_only && (t.cg0 + j > t.rg0 + i));
+                        v1[nf][h] = i < t.Mt && j + 1 < t.Nt && !(t.lower_only && (t.cg0 + j + 1 > t.rg0 + i));
+                        cv2[nf][h] = (v0[nf][h] && t.beta != 0.f) ? *reinterpret_cast<const float2*>(t.C + i * t.c_rs + j)
+                                                                  : make_float2(0.f, 0.f);
+                    }
+#pragma unroll
+                for (int nf = 0; nf < 4; ++nf)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int i = row0 + gq + h * 8, j = col0 + nf * 8 + tq * 2;
+                        const float o0 = fmaf(t.beta, cv2[nf][h].x, t.alpha * acc[nf][2 * h]);
+                        const float o1 = fmaf(t.beta, cv2[nf][h].y, t.alpha * acc[nf][2 * h + 1]);
+                        if (v0[nf][h] && v1[nf][h]) *reinterpret_cast<float2*>(t.C + i * t.c_rs + j) = make_float2(o0, o1);
+                        else if (v0[nf][h]) t.C[i * t.c_rs + j] = o0;
+                        acc[nf][2 * h] = 0.f; acc[nf][2 * h + 1] = 0.f;
+                    }
+            } else {
+            float cv[4][4];
+            bool valid[4][4];
+#pragma unroll
+            for (int nf = 0; nf < 4; ++nf)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = row0 + gq + (e / 2) * 8, j = col0 + nf * 8 + tq * 2 + (e % 2);
+                    valid[nf][e] = i < t.Mt && j < t.Nt && !(t.lower_only && (t.cg0 + j > t.rg0 + i));
+                    cv[nf][e] = (valid[nf][e] && t.beta != 0.f) ? t.C[i * t.c_rs + j * t.c_cs] : 0.f;
+                }
+#pragma unroll
+            for (int nf = 0; nf < 4; ++nf)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = row0 + gq + (e / 2) * 8, j = col0 + nf * 8 + tq * 2 + (e % 2);
+                    if (valid[nf][e]) t.C[i * t.c_rs + j * t.c_cs] = fmaf(t.beta, cv[nf][e], t.alpha * acc[nf][e]);
+                    acc[nf][e] = 0.f;
+                }
+            }
+        }
+        if (!has_next) break;
+        ti = nti; k0 = nk0;
+    }
+    __syncthreads();
+}
+
+// One warp: Cholesky of a 32 x 32 block held one row per lane (a[c], c <= lane; rows >= nb must be
+// identity rows).  On return a[] is the row of L.  Returns true if a pivot was not positive.
+__device__ __forceinline__ bool warp_chol32(float (&a)[32], int lane, int nb, float& dmin, float& dmax) {
+    bool fail = false;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        float d = __shfl_sync(0xffffffffu, a[j], j);
+        if (!(d > 0.f) || !(d <= 3.0e38f)) { if (j < nb) fail = true; d = 1.f; }
+        const float s = sqrtf(d);
+        if (j < nb) { dmin = fminf(dmin, s); dmax = fmaxf(dmax, s); }
+        const float lij = (lane > j) ? a[j] / s : 0.f;
+        if (lane == j) a[j] = s;
+        else if (lane > j) a[j] = lij;
+#pragma unroll
+        for (int c = j + 1; c < 32; ++c) {
+            const float lcj = __shfl_sync(0xffffffffu, lij, c);
+            if (lane >= c) a[c] = fmaf(-lij, lcj, a[c]);
+        }
+    }
+    return fail;
+}
+
+__global__ void __launch_bounds__(CT_THREADS, 2)
+chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
+    __shared__ __align__(16) __nv_bfloat16 s_stage[4 * 64 * CT_LDK];
+    __shared__ TcTask s_tasks[CT_MAX_TASKS];
+    __shared__ float s_diag[1024];
+    __shared__ float red[8];
+    __shared__ int s_ntasks, s_fail, s_status;
+    __shared__ float s_trace, s_dmin, s_dmax;
+
+    const MatWork& w = batch.w[blockIdx.x];
+    const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
+    const int r = a.r;
+    const int shift_bit = a.which ? ST_SHIFT_R : ST_SHIFT_L;
+
+    if (tid == 0) s_status = *w.status;
+    __syncthreads();
+    const int st0 = s_status;
+    if (st0 & ST_FAILED) return;
+    if (a.pass == 3 && !(st0 & shift_bit)) return;
+
+    const float* __restrict__ A = pick(w, a.gram);     // Gram matrix: never written here
+    float* W = pick(w, a.work);
+
+    // diagonal (from the fp32 column sums of squares), trace, finiteness
+    {
+        float t = 0.f;
+        for (int i = tid; i < r; i += CT_THREADS) {
+            float d;
+            if (a.use_colsq) {
+                const float* cs = pick(w, a.colsq);
+                d = 0.f;
+                for (int kb = 0; kb < w.aux0; ++kb) d += cs[kb * r + i];
+            } else {
+                d = A[i * r + i];
+            }
+            s_diag[i] = d;
+            if (a.cnorm_off >= 0) reinterpret_cast<float*>(w.scratch + a.cnorm_off)[i] = d;
+            t += d;
+        }
+        for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0) red[warp] = t;
+        __syncthreads();
+        if (tid == 0) {
+            float s = 0.f;
+            for (int i = 0; i < CT_THREADS / 32; ++i) s += red[i];
+            s_trace = s;
+        }
+        __syncthreads();
+    }
+    const float trace = s_trace;
+    if (!(fabsf(trace) <= 3.0e38f)) {   // Inf or NaN
+        if (tid == 0) atomicOr(w.status, ST_NONFINITE);
+        return;
+    }
+
+    auto add_task = [&](float* C, int c_rs, int c_cs, const float* A_, int a_rs, const float* B_, int b_rs, int b_cs,
+                        int Mt, int Nt, int kbeg, int kend, float alpha, float beta, bool lower_only, int rg0, int cg0) {
+        TcTask& t = s_tasks[s_ntasks++];
+        t.C = C; t.A = A_; t.B = B_;
+        t.c_rs = c_rs; t.c_cs = c_cs; t.a_rs = a_rs; t.b_rs = b_rs; t.b_cs = b_cs;
+        t.Mt = Mt; t.Nt = Nt; t.kbeg = kbeg; t.kend = kend; t.lower_only = lower_only ? 1 : 0; t.rg0 = rg0; t.cg0 = cg0;
+        t.alpha = alpha; t.beta = beta;
+    };
+
+    bool ok = false;
+    const int max_attempts = (a.pass == 1) ? 2 : 1;
+    for (int attempt = 0; attempt < max_attempts && !ok; ++attempt) {
+        const float shift = attempt ? a.shift_rel * trace : 0.f;
+        // W <- lower(A) + shift*I (diagonal from s_diag), strict upper part zero; 4 columns per thread
+        const int r4 = r / 4;
+        for (int q = tid; q < r * r4; q += CT_THREADS) {
+            const int i = q / r4, j4 = (q - i * r4) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (j4 <= i) {
+                v = *reinterpret_cast<const float4*>(A + i * r + j4);
+                if (j4 + 0 > i) v.x = 0.f; else if (j4 + 0 == i) v.x = s_diag[i] + shift;
+                if (j4 + 1 > i) v.y = 0.f; else if (j4 + 1 == i) v.y = s_diag[i] + shift;
+                if (j4 + 2 > i) v.z = 0.f; else if (j4 + 2 == i) v.z = s_diag[i] + shift;
+                if (j4 + 3 > i) v.w = 0.f; else if (j4 + 3 == i) v.w = s_diag[i] + shift;
+            }
+            *reinterpret_cast<float4*>(W + i * r + j4) = v;
+        }
+        if (tid == 0) { s_fail = 0; s_dmin = 3.0e38f; s_dmax = 0.f; }
+        __syncthreads();
+
+        for (int k0 = 0; k0 < r; k0 += CT_NB) {
+            const int nb = min(CT_NB, r - k0);
+            if (warp == 0) {
+                // factor the diagonal block and replace it by its inverse
+                float row[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    row[c] = (lane < nb && c <= lane) ? W[(k0 + lane) * r + k0 + c] : (c == lane ? 1.f : 0.f);
+                float dmin = 3.0e38f, dmax = 0.f;
+                const bool fail = warp_chol32(row, lane, nb, dmin, dmax);
+                // lane c solves L x = e_c (column c of the inverse); L(i, p) comes from lane i's registers
+                float x[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float sacc = (i == lane) ? 1.f : 0.f;
+#pragma unroll
+                    for (int p = 0; p < i; ++p) sacc = fmaf(-__shfl_sync(0xffffffffu, row[p], i), x[p], sacc);
+                    const float lii = __shfl_sync(0xffffffffu, row[i], i);
+                    x[i] = (i >= lane) ? sacc / lii : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < nb && lane < nb && i >= lane) W[(k0 + i) * r + k0 + lane] = x[i];
+                if (lane == 0) {
+                    if (fail) s_fail = 1;
+                    s_dmin = fminf(s_dmin, dmin);
+                    s_dmax = fmaxf(s_dmax, dmax);
+                }
+            }
+            __syncthreads();
+            const int t0 = k0 + nb, s = r - t0;
+            if (s > 0) {
+                // panel: rows below <- rows below * inv(L_kk)^T
+                if (tid == 0) {
+                    s_ntasks = 0;
+                    for (int i0 = 0; i0 < s; i0 += 64)
+                        add_task(W + (t0 + i0) * r + k0, r, 1, W + (t0 + i0) * r + k0, r, W + k0 * r + k0, 1, r,
+                                 min(64, s - i0), nb, 0, nb, 1.f, 0.f, false, 0, 0);
+                }
+                __syncthreads();
+                tc_run_tasks(s_tasks, s_ntasks, s_stage);
+                // trailing update: W[t0+i][t0+j] -= sum_c W[t0+i][k0+c] W[t0+j][k0+c], j <= i
+                if (tid == 0) {
+                    s_ntasks = 0;
+                    const int nt = (s + 63) / 64;
+                    for (int ti = 0; ti < nt; ++ti)
+                        for (int tj = 0; tj <= ti; ++tj) {
+                            const int ri = t0 + ti * 64, cj = t0 + tj * 64;
+                            add_task(W + ri * r + cj, r, 1, W + ri * r + k0, r, W + cj * r + k0, 1, r,
+                                     min(64, r - ri), min(64, r - cj), 0, nb, -1.f, 1.f, ti == tj, ri, cj);
+                        }
+                }
+                __syncthreads();
+                tc_run_tasks(s_tasks, s_ntasks, s_stage);
+            }
+        }
+        const bool fail = s_fail != 0;
+        const bool ill = (a.pass == 1) && (s_dmax > a.cond_limit * s_dmin);
+        if (!fail && !(ill && attempt == 0)) {
+            ok = true;
+        } else if (attempt == 0 && a.pass == 1) {
+            if (tid == 0) atomicOr(w.status, shift_bit);
+        }
+        __syncthreads();
+    }
+    if (!ok) {
+        if (tid == 0) atomicOr(w.status, ST_RANKDEF);
+        return;
+    }
+
+    // ---- inverse of the lower factor: the diagonal blocks are inverted already; combine pairwise
+    for (int s = CT_NB; s < r; s *= 2) {
+        const int npairs = (r + 2 * s - 1) / (2 * s);
+        // step 1: T = B * Ai, kept transposed in the (unused, zero) mirror block above the diagonal
+        if (tid == 0) {
+            s_ntasks = 0;
+            for (int pr = 0; pr < npairs; ++pr) {
+                const int p = pr * 2 * s, sc = min(s, r - p - s);
+                if (sc <= 0) continue;
+                for (int i0 = 0; i0 < sc; i0 += 64)
+                    for (int c0 = 0; c0 < s; c0 += 64)
+                        add_task(W + (p + c0) * r + (p + s + i0), 1, r,           // T(i,k) at W[p+k][p+s+i]
+                                 W + (p + s + i0) * r + p, r,                     // B(i,q)
+                                 W + p * r + (p + c0), r, 1,                      // Ai(q,k)
+                                 min(64, sc - i0), min(64, s - c0), c0, s, 1.f, 0.f, false, 0, 0);
+            }
+        }
+        __syncthreads();
+        tc_run_tasks(s_tasks, s_ntasks, s_stage);
+        // step 2: B <- -Ci * T
+        if (tid == 0) {
+            s_ntasks = 0;
+            for (int pr = 0; pr < npairs; ++pr) {
+                const int p = pr * 2 * s, sc = min(s, r - p - s);
+                if (sc <= 0) continue;
+                for (int i0 = 0; i0 < sc; i0 += 64)
+                    for (int c0 = 0; c0 < s; c0 += 64)
+                        add_task(W + (p + s + i0) * r + (p + c0), r, 1,           // Bnew(i,k)
+                                 W + (p + s + i0) * r + (p + s), r,               // Ci(i,q)
+                                 W + (p + c0) * r + (p + s), 1, r,                // T(q,k) at W[p+k][p+s+q]
+                                 min(64, sc - i0), min(64, s - c0), 0, min(sc, i0 + 64), -1.f, 0.f, false, 0, 0);
+            }
+        }
+        __syncthreads();
+        tc_run_tasks(s_tasks, s_ntasks, s_stage);
+        // clear the mirror blocks again
+        for (int pr = 0; pr < npairs; ++pr) {
+            const int p = pr * 2 * s, sc = min(s, r - p - s);
+            if (sc <= 0) continue;
+            for (int e = tid; e < s * sc; e += CT_THREADS) {
+                const int k = e / sc, i = e - k * sc;
+                W[(p + k) * r + (p + s + i)] = 0.f;
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- split image of L^{-1} for the tensor-core apply product ------------------------------
+    if (a.img.off >= 0) {
+        unsigned char* __restrict__ scr = reinterpret_cast<unsigned char*>(w.scratch);
+        const float* __restrict__ Wr = W;
+        const int chunks = a.img.panels * a.img.rows_pad * 8;
+        for (int q = tid; q < chunks; q += CT_THREADS) {
+            const int c = q % 8, row = (q / 8) % a.img.rows_pad, panel = q / (8 * a.img.rows_pad);
+            const int col = panel * 64 + c * 8;
+            float v[8];
+            if (row < r && col + 7 < r) {
+                const float4* p4 = reinterpret_cast<const float4*>(Wr + row * r + col);
+                const float4 x = p4[0], y = p4[1];
+                v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = (row < r && col + i < r) ? Wr[row * r + col + i] : 0.f;
+            }
+            uint4 t0, t1;
+            split8(v, t0, t1);
+            const int o = img_chunk_offset(row, c);
+            *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 0, panel, row) + o) = t0;
+            *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 1, panel, row) + o) = t1;
+        }
+    }
+}
+
+}  // namespace od

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "profile.cuh"
 #include "factor_kernels.cuh"
+#include "factor_tc.cuh"
 #include "simt_kernels.cuh"
 #include "tensor_engine.cuh"
 
@@ -195,7 +196,8 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
         auto flush = [&]() {
             if (!merged->count) return;
             prof::Scope scope(prof::S_CHOL, st);
-            chol_inv_kernel<<<merged->count, CH_THREADS, CH_SMEM_BYTES, st>>>(*merged, ca);
+            if (lead.tensor()) chol_inv_tc_kernel<<<merged->count, CT_THREADS, 0, st>>>(*merged, ca);
+            else chol_inv_kernel<<<merged->count, CH_THREADS, CH_SMEM_BYTES, st>>>(*merged, ca);
             merged->count = 0;
         };
         for (size_t j = i; j < which_cls.size(); ++j) {
