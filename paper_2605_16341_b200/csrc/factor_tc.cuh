@@ -211,9 +211,11 @@ __device__ __forceinline__ bool warp_chol32(float (&a)[32], int lane, int nb, fl
         if (lane == j) a[j] = s;
         else if (lane > j) a[j] = lij;
 #pragma unroll
-        for (int c = j + 1; c < 32; ++c) {
-            const float lcj = __shfl_sync(0xffffffffu, lij, c);
-            if (lane >= c) a[c] = fmaf(-lij, lcj, a[c]);
+        for (int c = 0; c < 32; ++c) {
+            if (c > j) {      // both loops run over the full range so that every index is a constant
+                const float lcj = __shfl_sync(0xffffffffu, lij, c);
+                if (lane >= c) a[c] = fmaf(-lij, lcj, a[c]);
+            }
         }
     }
     return fail;
@@ -320,7 +322,8 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
                 for (int i = 0; i < 32; ++i) {
                     float sacc = (i == lane) ? 1.f : 0.f;
 #pragma unroll
-                    for (int p = 0; p < i; ++p) sacc = fmaf(-__shfl_sync(0xffffffffu, row[p], i), x[p], sacc);
+                    for (int p = 0; p < 32; ++p)
+                        if (p < i) sacc = fmaf(-__shfl_sync(0xffffffffu, row[p], i), x[p], sacc);
                     const float lii = __shfl_sync(0xffffffffu, row[i], i);
                     x[i] = (i >= lane) ? sacc / lii : 0.f;
                 }
