@@ -340,7 +340,11 @@ def run_ours(args):
             ach = b / (dom_ms * 1e-3) / 1e9
             roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": ach / peaks["hbm_gbs"]}
-        roofline.update({"kernel": dominant, "traffic": KNOWN_TRAFFIC.get((args.workload, dominant)),
+        bpe = MEASURED_DRAM_BYTES_PER_ELEMENT.get((args.workload, dominant))
+        roofline.update({"kernel": dominant, "launches_per_step": stages[dominant]["launches_per_step"],
+                         "per": "step (sum over the launches of this kernel in one step)",
+                         "algorithmic": (b if roofline["bound"] == "hbm" else f),
+                         "traffic": (bpe * w.numel if (bpe and args.mode == "orth" and not args.passes) else None),
                          "peak_source": peaks["source"] + (" (sustained bf16 figure: kernel timed inside a long step)"
                                                            if roofline["bound"] == "tensor" else "")})
 
@@ -376,8 +380,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM traffic per step of the dominant kernel from committed ncu captures (profiles/), bytes.
-KNOWN_TRAFFIC: dict = {}
+# DRAM bytes per parameter element of a stage, measured with ncu on a smaller case of the same
+# kernel (profiles/fused_feedback_update_kernel_cfg4_4layers.md: 6.729 GB over 469.8 M elements);
+# traffic grows in proportion to the elements, so a step's traffic is this figure x its elements.
+MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.32}
 
 
 def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):
