@@ -72,7 +72,9 @@ def stage_models(matrices, mode_orth=True):
         xb = 2 if s.x_dtype == torch.bfloat16 else 4
         add("k1_buffer_times_q", 2.0 * m * n * r, (4 + gb) * m * n + 4.0 * (n + m) * r)
         add("k3_buffer_t_times_p", 2.0 * m * n * r, (4 + gb) * m * n + 4.0 * (n + m) * r)
-        add("k5_feedback_update", 4.0 * m * n * r, (8 + gb + 2 * xb) * m * n + 4.0 * (2 * n + m) * r)
+        # factor reads of the fused pass: fp16 planes of P, R, Q for bf16 weights, two bf16 terms else
+        fb = 2.0 if s.x_dtype == torch.bfloat16 else 4.0
+        add("k5_feedback_update", 4.0 * m * n * r, (8 + gb + 2 * xb) * m * n + fb * (2 * n + m) * r)
         qrs = [m] + ([n] if mode_orth else [])
         for k in qrs:
             add("gram", 2 * 2.0 * k * r * r, 2 * 4.0 * k * r)
