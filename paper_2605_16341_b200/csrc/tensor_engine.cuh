@@ -558,7 +558,9 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                         tc_fence_after();
                         if (lane == 0) {
                             const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
-                            const uint32_t ncols = (uint32_t)min(128, c.bn - ch * 128);
+                            // N of the instruction must be a multiple of 16: round a ragged last chunk up
+                            // (rows beyond the matrix are zero in the images; those columns of D are never stored)
+                            const uint32_t ncols = (uint32_t)((min(128, c.bn - ch * 128) + 15) / 16 * 16);
                             const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u, fmt);
                             for (int j = 0; j < nsl; ++j) {
                                 const uint64_t a0 = A_MN ? smem_desc(sa + j * 2048, 8192, 1024)
