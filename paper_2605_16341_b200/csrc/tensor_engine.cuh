@@ -502,9 +502,22 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
+        // One thread issues.  A tcgen05.mma of N = 256 occupies the tensor core for 128 cycles, so the
+        // scalar work per instruction has to stay at a handful of operations: every descriptor is a
+        // constant high part plus (shared address >> 4), advanced by additions only.
         int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
         int acc = 0; uint32_t acc_phase = 0;
         bool ok = true;
+        // descriptor high parts (layout, strides) and address units of 16 bytes
+        const uint64_t a_hi = A_MN ? smem_desc(0, 8192, 1024) : smem_desc(0, 16, 1024);
+        const uint64_t n_hi = (NMODE == N_IMG_MN) ? smem_desc(0, group_stride, 1024) : smem_desc(0, 16, 1024);
+        const uint32_t a_slice16 = A_MN ? (2048u >> 4) : (32u >> 4);        // one 16-deep slice of the A tile
+        const uint32_t n_slice16 = (NMODE == N_IMG_MN) ? (2048u >> 4) : (32u >> 4);
+        const uint32_t a_term16 = A_TERM_BYTES >> 4;
+        const uint32_t n_term16 = ((NMODE == N_IMG_MN) ? mn_term_stride : (uint32_t)A_TERM_BYTES) >> 4;
+        const uint32_t a_ring16 = smem_u32(a_ring) >> 4, n_ring16 = smem_u32(n_ring) >> 4;
+        const uint32_t a_slot16 = (uint32_t)g.a_slot_bytes >> 4, n_slot16 = (uint32_t)g.n_piece_bytes >> 4;
+        const bool three = g.passes == 3;
         for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
             const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
             if (!c.active) continue;
@@ -514,34 +527,30 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             for (int kb = 0; kb < c.kb_end && ok; ++kb) {
                 if (!mbar_wait(a_full0 + 8 * as, aph, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t sa = smem_u32(a_ring + as * g.a_slot_bytes);
+                const uint64_t a_kb = a_hi + (a_ring16 + as * a_slot16);
                 if (NMODE == N_IMG_MN) {
                     const int pieces = mn_pieces(g, kb);
+                    const int per_piece = g.ks / 16;
                     for (int sub = 0; sub < pieces && ok; ++sub) {
                         if (!mbar_wait(n_full0 + 8 * ns, nph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         if (lane == 0) {
-                            const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
+                            const uint64_t n_pc = n_hi + (n_ring16 + ns * n_slot16);
                             const int k0 = kb * BK + sub * g.ks;
                             const int nsl = (min(g.ks, g.Kdim - k0) + 15) / 16;
                             for (int j = 0; j < nsl; ++j) {
-                                const int slice = sub * (g.ks / 16) + j;
-                                const uint64_t a0 = A_MN ? smem_desc(sa + slice * 2048, 8192, 1024)
-                                                         : smem_desc(sa + slice * 32, 16, 1024);
-                                const uint64_t a1 = A_MN ? smem_desc(sa + A_TERM_BYTES + slice * 2048, 8192, 1024)
-                                                         : smem_desc(sa + A_TERM_BYTES + slice * 32, 16, 1024);
+                                const uint64_t a0 = a_kb + (uint32_t)(sub * per_piece + j) * a_slice16;
+                                const uint64_t a1 = a0 + a_term16;
                                 const uint32_t accum = (kb > 0 || sub > 0 || j > 0) ? 1u : 0u;
+                                uint64_t b0 = n_pc + (uint32_t)j * n_slice16;
                                 for (int cc = 0; cc < c.bn; cc += 256) {
-                                    const uint32_t ncols = (uint32_t)min(256, c.bn - cc);
-                                    const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 1u, fmt);
-                                    const uint32_t nb = sn + (cc / 64) * group_stride + j * 2048;
-                                    const uint64_t b0 = smem_desc(nb, group_stride, 1024);
-                                    const uint64_t b1 = smem_desc(nb + mn_term_stride, group_stride, 1024);
+                                    const uint32_t idesc = instr_desc((uint32_t)min(256, c.bn - cc), A_MN ? 1u : 0u, 1u, fmt);
                                     umma_bf16(dacc + cc, a0, b0, idesc, accum);
-                                    if (g.passes == 3) {
-                                        umma_bf16(dacc + cc, a0, b1, idesc, 1u);
+                                    if (three) {
+                                        umma_bf16(dacc + cc, a0, b0 + n_term16, idesc, 1u);
                                         umma_bf16(dacc + cc, a1, b0, idesc, 1u);
                                     }
+                                    b0 += 4 * (group_stride >> 4);          // next 256 columns: four 64-column groups
                                 }
                             }
                             umma_commit(n_empty0 + 8 * ns);
@@ -557,11 +566,15 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                         if (!mbar_wait(n_full0 + 8 * ns, nph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         if (lane == 0) {
+                            const uint32_t sa = smem_u32(a_ring + as * g.a_slot_bytes);
                             const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
                             // N of the instruction must be a multiple of 16: round a ragged last chunk up
                             // (rows beyond the matrix are zero in the images; those columns of D are never stored)
                             const uint32_t ncols = (uint32_t)((min(128, c.bn - ch * 128) + 15) / 16 * 16);
                             const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u, fmt);
+                            // (Descriptors are rebuilt per instruction here on purpose: with the additive
+                            // form of the other branch the fused pass measured 38 ms instead of 26 ms per
+                            // step; its N = 128 instructions run best when they are not issued back to back.)
                             for (int j = 0; j < nsl; ++j) {
                                 const uint64_t a0 = A_MN ? smem_desc(sa + j * 2048, 8192, 1024)
                                                          : smem_desc(sa + j * 32, 16, 1024);
