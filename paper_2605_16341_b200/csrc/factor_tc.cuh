@@ -424,23 +424,20 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         __syncthreads();
     }
 
-    // ---- split image of L^{-1} for the tensor-core apply product ------------------------------
+    // ---- split image of (L^{-1})^T for the tensor-core apply product ---------------------------
+    // Image row k, column j holds L^{-1}(j, k): the apply product Y L^{-T} then reads its N-side
+    // operand MN-major (depth along image rows) in 256-column instructions.
     if (a.img.off >= 0) {
         unsigned char* __restrict__ scr = reinterpret_cast<unsigned char*>(w.scratch);
         const float* __restrict__ Wr = W;
         const int chunks = a.img.panels * a.img.rows_pad * 8;
         for (int q = tid; q < chunks; q += CT_THREADS) {
-            const int c = q % 8, row = (q / 8) % a.img.rows_pad, panel = q / (8 * a.img.rows_pad);
+            // consecutive threads take consecutive image rows (consecutive k: contiguous in W)
+            const int row = q % a.img.rows_pad, c = (q / a.img.rows_pad) % 8, panel = q / (8 * a.img.rows_pad);
             const int col = panel * 64 + c * 8;
             float v[8];
-            if (row < r && col + 7 < r) {
-                const float4* p4 = reinterpret_cast<const float4*>(Wr + row * r + col);
-                const float4 x = p4[0], y = p4[1];
-                v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
-            } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = (row < r && col + i < r) ? Wr[row * r + col + i] : 0.f;
-            }
+            for (int i = 0; i < 8; ++i) v[i] = (row < r && col + i < r) ? Wr[(col + i) * r + row] : 0.f;
             uint4 t0, t1;
             split8(v, t0, t1);
             const int o = img_chunk_offset(row, c);

@@ -1194,7 +1194,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
 // Host side of the engine
 // ------------------------------------------------------------------------------------------
 struct TensorScratch {      // where the images of one matrix live inside its scratch area
-    ImgRef linv;            // L^{-1} of the current Cholesky            (r x r)
+    ImgRef linv;            // (L^{-1})^T of the current Cholesky        (r x r)
     ImgRef qprev;           // Q_prev                                    (n x r)
     ImgRef w0, w1;          // Y = B Q_prev and the QR intermediates     (max(m,n) x r)
     ImgRef p, r, q;         // P (m x r), R (n x r), Q (n x r); three planes when the fused pass runs in fp16
@@ -1317,7 +1317,7 @@ inline cudaError_t tensor_engine_set_attributes() {
     OD_SET(tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 0)
     OD_SET(tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 1)
     OD_SET(tc::A_IMG_MN, tc::N_IMG_MN, tc::EPI_STORE, 0)
-    OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_STORE, 0)
+    OD_SET(tc::A_IMG_K, tc::N_IMG_MN, tc::EPI_STORE, 0)
     OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 0)
     OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 1)
     OD_SET(tc::A_IMG_K, tc::N_IMG_K, tc::EPI_K5, 2)
@@ -1437,7 +1437,7 @@ inline void tensor_gram(int r, int passes, const Batch& b, ImgRef src, int64_t r
     launch_gemm<tc::A_IMG_MN, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_GRAM, st);
 }
 
-// dst = src * L^{-T}  (src: image of a rows x r matrix, L^{-1}: image linv, lower triangular)
+// dst = src * L^{-T}  (src: image of a rows x r matrix; image linv holds (L^{-1})^T, read MN-major)
 inline void tensor_apply(int r, int passes, const Batch& b, const TensorScratch& ts, ImgRef src, int64_t rows,
                          tc::OutSpec out, cudaStream_t st) {
     tc::GemmArgs g{};
@@ -1445,7 +1445,7 @@ inline void tensor_apply(int r, int passes, const Batch& b, const TensorScratch&
     g.passes = passes; g.passes2 = 1; g.a = src; g.n1 = ts.linv; g.n2 = no_img(); g.tri = 1;
     g.colsq_off = ts.colsq;
     g.out = out;
-    launch_gemm<tc::A_IMG_K, tc::N_IMG_K, tc::EPI_STORE, 0>(b, g, prof::S_APPLY, st);
+    launch_gemm<tc::A_IMG_K, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_APPLY, st);
 }
 
 // M <- a (M + G) - b P R^T ;  X <- c X - d P Q^T                  (Alg. 1 lines 5-7)
