@@ -4,18 +4,18 @@
  * paper ("Orth-Dion / Stripped Dion (one step)"; appendix algorithms "Stripped Dion" and
  * "Orth-Dion"), written with the letters of this interface:
  *
- *     B  = M + G                                 buffer            (Alg. 1 line 1)
- *     P  = orth(B * Q_prev)                      left factor       (Alg. 1 line 2)
- *     R  = B^T * P                               right factor      (Alg. 1 line 3)
- *     Q  = orth(R)   [ORTH]   |  ColNorm(R) [COLNORM]              (Alg. 1 line 4)
- *     X <- (1 - eta*wd) * X - eta*scale * P * Q^T                  (Alg. 1 lines 5-6)
- *     M <- a * B - b * P * R^T                   error feedback    (Alg. 1 line 7)
- *     Q_prev <- Q                                warm start        (Alg. 1 line 8)
+ *     B  = M + G                                 buffer            (Alg. 1, buffer step)
+ *     P  = orth(B * Q_prev)                      left factor       (Alg. 1, left-factor step)
+ *     R  = B^T * P                               right factor      (Alg. 1, right-factor step)
+ *     Q  = orth(R)   [ORTH]   |  ColNorm(R) [COLNORM]              (Alg. 1, normalisation step)
+ *     X <- (1 - eta*wd) * X - eta*scale * P * Q^T                  (Alg. 1, update step)
+ *     M <- a * B - b * P * R^T                   error feedback    (Alg. 1, error-feedback step)
+ *     Q_prev <- Q                                warm start        (Alg. 1, warm-start step)
  *
  * Paper letters: G_t = G, R_t = M (residual), M_t = B, V_{t-1} = Q_prev, U_t = P, W_t = R.
  * orth(.) is the thin QR factor with a positive diagonal in the triangular factor
  * (CholeskyQR2 on the device, with a shifted third pass when the Gram matrix is
- * ill-conditioned).  (a, b) default to (1, 1 - mu); the paper's line 7 is (beta, beta).
+ * ill-conditioned).  (a, b) default to (1, 1 - mu); the paper's error-feedback step is (beta, beta).
  *
  * Conventions
  *  - Every matrix pointer is a DEVICE pointer owned by the caller; matrices are row-major and
@@ -47,7 +47,7 @@ extern "C" {
 
 typedef struct orthdion_plan* orthdion_t;
 
-/* Algorithm 1 line 4: which normalisation of the right factor. */
+/* Algorithm 1, normalisation step: which normalisation of the right factor. */
 #define ORTHDION_MODE_ORTH     0   /* Q = orth(R): Orth-Dion                     */
 #define ORTHDION_MODE_COLNORM  1   /* Q = ColNorm(R): (Stripped) Dion            */
 
@@ -77,7 +77,7 @@ typedef struct orthdion_plan* orthdion_t;
 #define ORTHDION_STATUS_ZERO_COLUMN    16   /* COLNORM met a zero column of R (kept zero)       */
 #define ORTHDION_STATUS_WAIT_LIMIT     32   /* a bounded device-side wait expired (kernel bug)  */
 
-/* Create a plan for m x n matrices at rank r (Algorithm 1 "REQUIRE" line: step size eta, EF
+/* Create a plan for m x n matrices at rank r (inputs of Algorithm 1: step size eta, EF
  * coefficient; mu gives the default (a, b) = (1, 1 - mu)).  Defaults: X and G bfloat16,
  * scale = 1, engine TENSOR.  The TENSOR engine needs r % 16 == 0, n % 8 == 0; SIMT any r.
  * Host memory only. */
@@ -158,8 +158,8 @@ int64_t orthdion_launch_count(void);
  * max_launches launches are recorded; profile_begin creates the events).  profile_end waits for
  * the recorded events and returns, per stage s < orthdion_stage_count(), the summed device time
  * ms[s] in milliseconds and the number of launches.  Stages are the kernels of the step: the
- * packers, Y = B*Q_prev (Alg. 1 line 2), Gram, Cholesky+inverse, apply (the QR of lines 2 and 4),
- * R = B^T*P (line 3), ColNorm (line 4) and the fused feedback/update pass (lines 5-7).
+ * packers, Y = B*Q_prev, Gram, Cholesky+inverse, apply (the QR of the left-factor and normalisation steps),
+ * R = B^T*P, ColNorm and the fused feedback/update pass.
  * Not thread-safe; meant for benchmarks. */
 int orthdion_profile_begin(int32_t max_launches);
 int orthdion_profile_end(int32_t n_stages, double* ms, int64_t* launches);

@@ -22,7 +22,7 @@ a Householder factorisation written out below.
 
 Parity pins: every function here is pinned by tests/test_oracle_pins.py against
 identities the paper states (Lemma 4.1, Prop. 3.1, Lemma 4.2, Lemma 4.3, the
-error-feedback line of Algorithm 1), closed forms, LAPACK QR / SVD, and the worked
+error-feedback step of Algorithm 1), closed forms, LAPACK QR / SVD, and the worked
 numbers the paper prints.  The weight-decay and scale factors of `step` have no
 equation in the paper: for wd != 0 or scale != 1 the parity is UNPINNED beyond the
 algebraic identity X' - (1 - eta*wd) X = -eta*scale*P Q^T.
@@ -31,8 +31,8 @@ from __future__ import annotations
 
 import numpy as np
 
-ORTH = 0      # Algorithm 1 line 4, Orth-Dion branch: QR of the right factor
-COLNORM = 1   # Algorithm 1 line 4, Dion branch: unit-length columns
+ORTH = 0      # Algorithm 1, normalisation step, Orth-Dion branch: QR of the right factor
+COLNORM = 1   # Algorithm 1, normalisation step, Dion branch: unit-length columns
 
 STATUS_OK = 0
 STATUS_RANK_DEFICIENT = 1   # a triangular factor has a (relatively) vanishing pivot
@@ -42,7 +42,7 @@ RANK_TOL = 1e-12
 
 
 # ----------------------------------------------------------------------------------
-# orth(.) : thin QR with positive diagonal  (Section 2, "orth(W_t) (QR)"; Alg. 1 l.2, l.4)
+# orth(.) : thin QR with positive diagonal  (Section 2, "orth(W_t) (QR)"; Alg. 1, left-factor and normalisation steps)
 # ----------------------------------------------------------------------------------
 def thin_qr_pos(Y: np.ndarray):
     """Thin QR factorisation Y = F T by Householder reflections, diag(T) > 0.
@@ -93,7 +93,7 @@ def thin_qr_pos(Y: np.ndarray):
 
 
 def col_norm(R: np.ndarray):
-    """ColNorm(W): every column scaled to unit Euclidean length (Section 3; Alg. 1 l.4, Dion).
+    """ColNorm(W): every column scaled to unit Euclidean length (Section 3; Alg. 1, normalisation step, Dion).
 
     Returns (Q, norms).  A zero column stays zero (its norm is reported as 0)."""
     R = np.asarray(R, dtype=np.float64)
@@ -110,9 +110,9 @@ def step(X, M, G, Qp, *, eta, mode=ORTH, mu=None, ef=None, wd=0.0, scale=1.0):
 
     Error feedback: M' = a*B - b*P R^T.
       * `mu` given  ->  (a, b) = (1, 1 - mu)        the momentum form M <- B - (1-mu) P R^T
-      * `ef=(a,b)`  ->  explicit; the paper's line 7, R_{t+1} = beta (M_t - U_t U_t^T M_t),
+      * `ef=(a,b)`  ->  explicit; the paper's error-feedback step, R_{t+1} = beta (M_t - U_t U_t^T M_t),
                         is ef=(beta, beta).
-    Weight update: X' = (1 - eta*wd) X - eta*scale * P Q^T   (Alg. 1 l.5-6 has wd=0, scale=1).
+    Weight update: X' = (1 - eta*wd) X - eta*scale * P Q^T   (Alg. 1, update step, has wd=0, scale=1).
     If a triangular factor is numerically singular the state is returned unchanged and
     status = STATUS_RANK_DEFICIENT (the paper assumes full rank)."""
     if (mu is None) == (ef is None):
@@ -123,22 +123,22 @@ def step(X, M, G, Qp, *, eta, mode=ORTH, mu=None, ef=None, wd=0.0, scale=1.0):
     G = np.asarray(G, dtype=np.float64)
     Qp = np.asarray(Qp, dtype=np.float64)
 
-    B = M + G                                   # Alg. 1 l.1   buffer
+    B = M + G                                   # Alg. 1, buffer step
     Y = B @ Qp
-    P, T1 = thin_qr_pos(Y)                      # Alg. 1 l.2   left factor
+    P, T1 = thin_qr_pos(Y)                      # Alg. 1, left-factor step
     status = STATUS_OK
     if _deficient(T1):
         status = STATUS_RANK_DEFICIENT
-    R = B.T @ P                                 # Alg. 1 l.3   right factor, un-normalised
+    R = B.T @ P                                 # Alg. 1, right-factor step (un-normalised)
     T2 = None
     colnorms = None
     if status == STATUS_OK:
         if mode == ORTH:
-            Q, T2 = thin_qr_pos(R)              # Alg. 1 l.4   Orth-Dion
+            Q, T2 = thin_qr_pos(R)              # Alg. 1, normalisation step: Orth-Dion
             if _deficient(T2):
                 status = STATUS_RANK_DEFICIENT
         elif mode == COLNORM:
-            Q, colnorms = col_norm(R)           # Alg. 1 l.4   Dion
+            Q, colnorms = col_norm(R)           # Alg. 1, normalisation step: Dion
             if np.any(colnorms == 0.0):
                 status = STATUS_ZERO_COLUMN
         else:
@@ -146,9 +146,9 @@ def step(X, M, G, Qp, *, eta, mode=ORTH, mu=None, ef=None, wd=0.0, scale=1.0):
     if status == STATUS_RANK_DEFICIENT:
         return dict(X=X.copy(), M=M.copy(), Q=Qp.copy(), P=P, R=R, T1=T1, T2=T2, B=B,
                     Y=Y, colnorms=colnorms, status=status)
-    D = P @ Q.T                                 # Alg. 1 l.5   update direction
-    Xn = (1.0 - eta * wd) * X - (eta * scale) * D   # Alg. 1 l.6
-    Mn = a * B - b * (P @ R.T)                  # Alg. 1 l.7   error feedback (P R^T = P P^T B)
+    D = P @ Q.T                                 # Alg. 1, update step: direction
+    Xn = (1.0 - eta * wd) * X - (eta * scale) * D   # Alg. 1, update step
+    Mn = a * B - b * (P @ R.T)                  # Alg. 1, error-feedback step (P R^T = P P^T B)
     return dict(X=Xn, M=Mn, Q=Q, P=P, R=R, T1=T1, T2=T2, B=B, Y=Y, D=D,
                 colnorms=colnorms, status=status)
 

@@ -350,7 +350,7 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     }
 }
 
-// ---- ColNorm (Alg. 1 line 4, Dion branch): Q[:,j] = R[:,j] / ||R[:,j]||_2 ----------------------
+// ---- ColNorm (Alg. 1, normalisation step, Dion branch): Q[:,j] = R[:,j] / ||R[:,j]||_2 ----------------------
 // One CTA per 32 columns: 32 x 32 threads, lanes along columns (coalesced rows).
 __global__ void __launch_bounds__(1024)
 colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t cnorm_off) {

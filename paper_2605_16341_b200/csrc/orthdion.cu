@@ -217,7 +217,7 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
 }
 
 // ---- tall-skinny QR of every class in `which_cls` (CholeskyQR2; third pass when flagged) --------
-// which = 0: P = orth(Y) (Alg. 1 line 2), which = 1: Q = orth(R) (Alg. 1 line 4).
+// which = 0: P = orth(Y) (Alg. 1, left-factor step), which = 1: Q = orth(R) (Alg. 1, normalisation step).
 // Tensor engine: the input is an image (w0 holds Y, image r holds R); SIMT engine: fp32 slots.
 void qr_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int which, Batch* merged,
               cudaStream_t st) {
@@ -289,7 +289,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
         prof::Scope scope(prof::S_MISC, st);
         init_status_kernel<<<(c.b->count + 255) / 256, 256, 0, st>>>(*c.b);
     }
-    // Alg. 1 lines 1-2:  Y = (M + G) Q_prev
+    // Alg. 1, buffer and left-factor steps:  Y = (M + G) Q_prev
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
         const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
@@ -298,7 +298,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
                          EpStore{sP, sP, 0, 0, p->r, 0}, prof::S_K1, st);
     }
     qr_stage(cls, all, 0, merged, st);
-    // Alg. 1 line 3:  R = (M + G)^T P
+    // Alg. 1, right-factor step:  R = (M + G)^T P
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
         const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
@@ -306,7 +306,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
         else launch_simt(*c.b, p->n, p->r, p->m, RdBuffer{p->n, gb, 1}, RdPlain{sP, 1, p->r},
                          EpStore{sR, sR, 0, 0, p->r, 0}, prof::S_K3, st);
     }
-    // Alg. 1 line 4
+    // Alg. 1, normalisation step
     qr_stage(cls, orth, 1, merged, st);
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
@@ -318,7 +318,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
         }
         if (c.tensor()) launch_pack(*c.b, sQ, p->n, p->r, c.sc.ts.q, st);
     }
-    // Alg. 1 lines 5-7:  M <- a B - b P R^T ;  X <- c X - d P Q^T
+    // Alg. 1, update and error-feedback steps:  M <- a B - b P R^T ;  X <- c X - d P Q^T
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
         const int gb = p->g_dtype == ORTHDION_DTYPE_BF16, xb = p->x_dtype == ORTHDION_DTYPE_BF16;

@@ -11,7 +11,7 @@ struct RdPlain {            // fp32 matrix with arbitrary strides: elem(i,k) = p
     static constexpr bool kBuf = false;
     __device__ __forceinline__ const float* base(const MatWork& w) const { return pick(w, sel); }
 };
-struct RdBuffer {           // B = M + G formed on the fly (Alg. 1 line 1); trans: elem(i,k)=B[k][i]
+struct RdBuffer {           // B = M + G formed on the fly (Alg. 1, buffer step); trans: elem(i,k)=B[k][i]
     int64_t ld; int32_t g_bf16; int32_t trans;
     static constexpr bool kBuf = true;
 };
@@ -42,7 +42,7 @@ struct EpStore {            // C[i*ld + j] = acc ; destination may depend on the
         c[i * ld + j] = acc;
     }
 };
-struct EpErrorFeedback {    // M <- a*(M+G) - b*acc          (Alg. 1 line 7)
+struct EpErrorFeedback {    // M <- a*(M+G) - b*acc          (Alg. 1, error-feedback step)
     float a, b; int64_t ld; int32_t g_bf16;
     __device__ __forceinline__ bool active(const MatWork& w) const { return !(*w.status & ST_FAILED); }
     __device__ __forceinline__ void operator()(const MatWork& w, int64_t i, int64_t j, float acc) const {
@@ -51,7 +51,7 @@ struct EpErrorFeedback {    // M <- a*(M+G) - b*acc          (Alg. 1 line 7)
         w.M[idx] = a * bval - b * acc;
     }
 };
-struct EpWeights {          // X <- c*X - d*acc              (Alg. 1 lines 5-6)
+struct EpWeights {          // X <- c*X - d*acc              (Alg. 1, update step)
     float c, d; int64_t ld; int32_t x_bf16;
     __device__ __forceinline__ bool active(const MatWork& w) const { return !(*w.status & ST_FAILED); }
     __device__ __forceinline__ void operator()(const MatWork& w, int64_t i, int64_t j, float acc) const {

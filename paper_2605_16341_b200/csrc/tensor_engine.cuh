@@ -9,7 +9,7 @@
 // matrices of the launch batch) drops into an operand ring, usable both K-major and MN-major,
 // so no kernel ever transposes.  Images are written by the epilogue of the kernel
 // that produces the matrix; only Q_prev (caller-owned fp32) is packed by a kernel of its own.
-// The big operand B = M + G (Alg. 1 line 1) is never stored: transform warps read M and G from
+// The big operand B = M + G (Alg. 1, buffer step) is never stored: transform warps read M and G from
 // HBM, add, split and write the A tile directly.
 //
 // One CTA per SM walks a tile list.  Two rings in shared memory: A tiles of 128 x 64 (both terms,
@@ -353,12 +353,12 @@ __device__ __forceinline__ bool k_piece_active(const GemmArgs& g, const TileCoor
 //   last 16       transform warps (A_BUF_* only): form B = M + G, split, write the A tile
 // AMODE  where the A tile comes from and how it lies in shared memory
 //          A_IMG_K / A_IMG_MN   image tile, K-major / MN-major
-//          A_BUF_ROW            rows of B = M + G      (K-major;  Y = B Q_prev, Alg. 1 line 2)
-//          A_BUF_COL            columns of B = M + G   (MN-major; R = B^T P,    Alg. 1 line 3)
+//          A_BUF_ROW            rows of B = M + G      (K-major;  Y = B Q_prev, Alg. 1, left-factor step)
+//          A_BUF_COL            columns of B = M + G   (MN-major; R = B^T P,    Alg. 1, right-factor step)
 // NMODE  N_IMG_K   pieces = 128-row chunks of the N range, 64 deep (image K-major)
 //        N_IMG_MN  pieces = ks-deep slices of the whole N range (image MN-major)
 // EPI    EPI_STORE  fp32 copy and/or split image (+ column-square partials) of D
-//        EPI_K5     M <- a (M+G) - b D1,  X <- c X - d D2     (Alg. 1 lines 5-7), D1 = P R^T, D2 = P Q^T
+//        EPI_K5     M <- a (M+G) - b D1,  X <- c X - d D2     (Alg. 1, update and error-feedback steps), D1 = P R^T, D2 = P Q^T
 // XG     bit 0: G is bf16, bit 1: X is bf16
 // ------------------------------------------------------------------------------------------
 template <int XG>
@@ -1069,7 +1069,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             }
         }
     } else if (A_BUF) {
-        // ---------------- transform warps: A tile of B = M + G (Alg. 1 line 1) ----------------
+        // ---------------- transform warps: A tile of B = M + G (Alg. 1, buffer step) ----------------
         // 512 threads, two 8-element chunks each per 128 x 64 tile; the loads of the next two
         // tiles are in flight while the current one is split and stored.
         const int xt = threadIdx.x - 32 * (2 + NE);     // 0 .. 511
@@ -1397,7 +1397,7 @@ inline tc::Dest dest_none() {
     return d;
 }
 
-// Y = (M + G) Q_prev  -> image w0 (+ column squares)              (Alg. 1 lines 1-2)
+// Y = (M + G) Q_prev  -> image w0 (+ column squares)              (Alg. 1, buffer and left-factor steps)
 inline void tensor_k1(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
                       cudaStream_t st) {
     launch_pack(b, Sel{W_Q, 0, 0}, n, r, ts.qprev, st);
@@ -1411,7 +1411,7 @@ inline void tensor_k1(int64_t m, int64_t n, int r, int g_bf16, int passes, const
     else launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K1, st);
 }
 
-// R = (M + G)^T P  -> fp32 R slot, image r (+ column squares)     (Alg. 1 line 3)
+// R = (M + G)^T P  -> fp32 R slot, image r (+ column squares)     (Alg. 1, right-factor step)
 inline void tensor_k3(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
                       cudaStream_t st) {
     tc::GemmArgs g{};
@@ -1448,7 +1448,7 @@ inline void tensor_apply(int r, int passes, const Batch& b, const TensorScratch&
     launch_gemm<tc::A_IMG_K, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_APPLY, st);
 }
 
-// M <- a (M + G) - b P R^T ;  X <- c X - d P Q^T                  (Alg. 1 lines 5-7)
+// M <- a (M + G) - b P R^T ;  X <- c X - d P Q^T                  (Alg. 1, update and error-feedback steps)
 // fp16 = 1: both products run as one fp16 pass from the fp16 planes of P, R, Q (R's plane must
 // have been written by launch_pack_half).
 inline void tensor_k5(int64_t m, int64_t n, int r, int g_bf16, int x_bf16, int passes_m, int passes_x, int fp16,

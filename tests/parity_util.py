@@ -1,5 +1,5 @@
 """Helpers for the GPU-vs-oracle parity tests: run the CUDA library and the float64 oracle on the
-same seeded tensors and compare what the benchmark spec's tolerance is stated on."""
+same seeded tensors and compare the quantities the tolerances are stated on."""
 from __future__ import annotations
 
 import numpy as np

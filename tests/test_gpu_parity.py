@@ -1,6 +1,6 @@
 """GPU-vs-oracle parity of the optimizer step, through the C-ABI, element by element.
 
-Tolerances (the benchmark spec): one step from identical state  ||dX_gpu - dX_or||_F / ||dX_or||_F <= 1e-4,
+Tolerances: one step from identical state  ||dX_gpu - dX_or||_F / ||dX_or||_F <= 1e-4,
 <= 1e-3 after 10 chained steps (GPU carries its own fp32 M, Q; the oracle float64), and
 max |Q^T Q - I| <= 1e-5.
 """

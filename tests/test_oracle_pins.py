@@ -125,7 +125,7 @@ def test_update_direction_norms(mode):
         assert 1.0 + 1e-6 < v <= np.sqrt(r)
 
 
-# ------------------------------------------------------------------ error feedback (Alg. 1 l.7)
+# ------------------------------------------------------------------ error feedback (Alg. 1, error-feedback step)
 def test_error_feedback_identities():
     X, M, G, Qp = problem(2)
     mu = 0.95
