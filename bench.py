@@ -234,6 +234,8 @@ def run_ours(args):
             if args.passes:
                 for which, pv in enumerate(int(x) for x in args.passes.split(",")):
                     od.orthdion_set_passes(h, which, pv)
+            if args.diagnostics:
+                od.orthdion_set_diagnostics(h, args.diagnostics)
             plan_cache[key] = h
         hs.append(plan_cache[key])
         X, M, Q = wl.initial_state(spec, seed, i, device=dev)
@@ -285,6 +287,14 @@ def run_ours(args):
     flags = od.orthdion_last_status(hs, ws, stream)
     failed = sum(1 for f in flags if f & (od.STATUS_RANK_DEFICIENT | od.STATUS_NONFINITE | od.STATUS_WAIT_LIMIT))
     shifted = sum(1 for f in flags if f & (od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT))
+    diag_summary = None
+    if args.diagnostics:
+        ds = [d for d in od.orthdion_last_diagnostics(hs, ws, stream) if d["nu"] == d["nu"]]
+        if ds:
+            diag_summary = {"nu_min": min(d["nu"] for d in ds), "nu_max": max(d["nu"] for d in ds),
+                            "erank_mean": sum(d["erank"] for d in ds) / len(ds),
+                            "eig_products_max": max(d["iterations"] for d in ds),
+                            "eig_products_mean": sum(d["iterations"] for d in ds) / len(ds)}
 
     # elements stepped by the whole job: N replicas (weak) or the one model split N ways (strong)
     elements = w.numel * world if args.scaling == "weak" else sum(s.numel for s in all_matrices)
@@ -364,7 +374,8 @@ def run_ours(args):
         "config": {"workload": f"{w.name}: {len(w.matrices)} matrices per rank, {elements / 1e6:.1f}M elements in the job, r={w.matrices[0].r}, "
                                f"bf16 X/G, fp32 M, mode {args.mode}",
                    "engine": args.engine, "l2": "inputs (tens of GB per step) far exceed the 126 MB L2",
-                   "grad_sets": args.grad_sets, "replicas": world,
+                   "grad_sets": args.grad_sets, "replicas": world, "diagnostics": args.diagnostics,
+                   "diagnostics_summary": diag_summary,
                    "matrices_failed": failed, "matrices_shifted_qr": shifted},
         "clocks": clocks,
         "e2e": e2e,
@@ -444,6 +455,8 @@ def main():
     ap.add_argument("--engine", default="tensor", choices=["tensor", "simt"])
     ap.add_argument("--passes", default=None,
                     help="bf16 split passes of the four product groups, e.g. 3,3,3,1 (0 keeps the default)")
+    ap.add_argument("--diagnostics", type=int, default=0, choices=[0, 1, 3],
+                    help="on-device diagnostics inside the timed step (0 off, 1 factor diagnostics, 3 plus buffer norms)")
     ap.add_argument("--grad-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")

@@ -26,7 +26,8 @@
  *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
  *    synchronising.  The library allocates no device memory: the caller passes a workspace of
  *    at least orthdion_workspace_bytes*() bytes, 256-byte aligned, which must stay untouched
- *    until the enqueued work has finished.  P, R and the status words live in it.
+ *    until the enqueued work has finished.  P, R, the status words and the
+ *    diagnostic records live in it.
  *  - Return value: 0 on success, a negative ORTHDION_ERR_* code when the host rejects the
  *    arguments (nothing is enqueued then).  Numerical conditions never trap: they are reported
  *    per matrix through status flags in the workspace (orthdion_last_status).  A matrix whose
@@ -149,6 +150,30 @@ int orthdion_get_factors(const orthdion_t* hs, int32_t count, int32_t index, voi
 /* Copies the `count` status words of the last step to host `flags` (synchronises `stream`). */
 int orthdion_last_status(const orthdion_t* hs, int32_t count, void* workspace, void* stream,
                          int32_t* flags);
+
+/* Optional per-step diagnostics (the paper's per-iteration quantities, appendix "Norms and Key
+ * Quantities", and the effective-rank estimator of the adaptive-rank section), computed on the
+ * device at the end of a step from what the step leaves behind.  mask: 0 off (default),
+ * 1 factor diagnostics, 3 factor diagnostics and buffer norms (one more read of M and G).
+ * Part of the plan's class: matrices with different masks are not batched together.
+ * orthdion_last_diagnostics copies ORTHDION_DIAG_FLOATS floats per matrix to host `out`
+ * (count * ORTHDION_DIAG_FLOATS floats; synchronises `stream`), in this order:
+ *   [0] nu      = ||Q||_op (Proposition 3.1: 1 for ORTH, in [1, sqrt(r)] for COLNORM), the root of
+ *                 the largest eigenvalue of Q^T Q by Lanczos iteration (at most 96 products with
+ *                 Q^T Q; stops once the top Ritz value has settled to 1e-6)
+ *   [1] erank   = exp(-sum_j p_j log p_j), p_j = ||R_j||_2 / sum_k ||R_k||_2
+ *   [2] tr_t2   = <B, P Q^T> = <R, Q>  (Lemma 4.2; tr(T_2) for ORTH, sum of column norms for COLNORM)
+ *   [3] norm_r  = ||R||_F = ||P^T B||_F
+ *   [4] norm_m  = ||M'||_F   [5] norm_g = ||G||_F   (mask 3 only, else 0)
+ *   [6] norm_b  = ||B||_F derived from ||M'||^2 = a^2 ||B||^2 - (2ab - b^2) ||R||^2, which holds
+ *                 when P^T P = I (mask 3 only, else 0; 0 when a = 0)
+ *   [7] number of products with Q^T Q the eigenvalue iteration used
+ * A matrix whose step failed (ORTHDION_STATUS_RANK_DEFICIENT or _NONFINITE) reports NaN in every
+ * slot; a matrix whose plan has diagnostics off reports zeros. */
+#define ORTHDION_DIAG_FLOATS 8
+int orthdion_set_diagnostics(orthdion_t h, int32_t mask);
+int orthdion_last_diagnostics(const orthdion_t* hs, int32_t count, void* workspace, void* stream,
+                              float* out);
 
 /* Number of kernels this library has launched so far in this process (monotonic). */
 int64_t orthdion_launch_count(void);

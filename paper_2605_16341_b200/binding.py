@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
     L.orthdion_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.orthdion_get_factors.argtypes = [pvp, i32, i32, vp, pvp, pvp]
     L.orthdion_last_status.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(i32)]
+    L.orthdion_set_diagnostics.argtypes = [vp, i32]
+    L.orthdion_last_diagnostics.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(ctypes.c_float)]
     L.orthdion_version.restype = ctypes.c_char_p
     L.orthdion_launch_count.restype = i64
     L.orthdion_profile_begin.argtypes = [i32]
@@ -87,7 +89,8 @@ def lib() -> ctypes.CDLL:
     L.orthdion_stage_name.argtypes = [i32]
     L.orthdion_stage_name.restype = ctypes.c_char_p
     for name in ("create", "destroy", "set_dtypes", "set_lr", "set_scale", "set_ef", "set_engine",
-                 "set_passes", "step", "step_grouped", "step_noalloc", "get_factors", "last_status"):
+                 "set_passes", "step", "step_grouped", "step_noalloc", "get_factors", "last_status",
+                 "set_diagnostics", "last_diagnostics"):
         getattr(L, "orthdion_" + name).restype = i32
     _lib = L
     return L
@@ -96,7 +99,8 @@ def lib() -> ctypes.CDLL:
 EXPORTED = ["orthdion_create", "orthdion_destroy", "orthdion_set_dtypes", "orthdion_set_lr",
             "orthdion_set_scale", "orthdion_set_ef", "orthdion_set_engine", "orthdion_set_passes",
             "orthdion_workspace_bytes", "orthdion_workspace_bytes_grouped", "orthdion_step",
-            "orthdion_step_grouped", "orthdion_step_noalloc", "orthdion_get_factors", "orthdion_last_status", "orthdion_version",
+            "orthdion_step_grouped", "orthdion_step_noalloc", "orthdion_get_factors", "orthdion_last_status",
+            "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_version",
             "orthdion_launch_count", "orthdion_profile_begin", "orthdion_profile_end", "orthdion_stage_count",
             "orthdion_stage_name"]
 
@@ -239,6 +243,22 @@ def orthdion_last_status(hs, workspace, stream=None):
     _check(lib().orthdion_last_status(_harr(hs), len(hs), _dev_ptr(workspace, "workspace"),
                                       _stream_ptr(stream), flags), "orthdion_last_status")
     return list(flags)
+
+
+DIAG_FLOATS = 8
+DIAG_NAMES = ("nu", "erank", "tr_t2", "norm_r", "norm_m", "norm_g", "norm_b", "iterations")
+
+
+def orthdion_set_diagnostics(h, mask: int):
+    _check(lib().orthdion_set_diagnostics(h, mask), "orthdion_set_diagnostics")
+
+
+def orthdion_last_diagnostics(hs, workspace, stream=None):
+    """One dict per matrix (keys DIAG_NAMES) from the diagnostic records of the last step."""
+    out = (ctypes.c_float * (DIAG_FLOATS * len(hs)))()
+    _check(lib().orthdion_last_diagnostics(_harr(hs), len(hs), _dev_ptr(workspace, "workspace"),
+                                           _stream_ptr(stream), out), "orthdion_last_diagnostics")
+    return [dict(zip(DIAG_NAMES, out[i * DIAG_FLOATS:(i + 1) * DIAG_FLOATS])) for i in range(len(hs))]
 
 
 def orthdion_launch_count() -> int:

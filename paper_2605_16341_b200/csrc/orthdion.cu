@@ -12,6 +12,7 @@
 #include "profile.cuh"
 #include "factor_kernels.cuh"
 #include "factor_tc.cuh"
+#include "diag_kernels.cuh"
 #include "simt_kernels.cuh"
 #include "tensor_engine.cuh"
 
@@ -24,6 +25,7 @@ struct orthdion_plan {
     float mu, eta, wd, scale, ef_a, ef_b;
     int32_t mode, x_dtype, g_dtype, engine;
     int32_t passes[4];
+    int32_t diag;          // bit 0: factor diagnostics, bit 1: buffer norms (extra sweep over M, G)
 };
 
 namespace {
@@ -41,7 +43,8 @@ bool same_class(const orthdion_plan* a, const orthdion_plan* b) {
     return a->m == b->m && a->n == b->n && a->r == b->r && a->mode == b->mode &&
            a->x_dtype == b->x_dtype && a->g_dtype == b->g_dtype && a->engine == b->engine &&
            a->eta == b->eta && a->wd == b->wd && a->scale == b->scale && a->ef_a == b->ef_a &&
-           a->ef_b == b->ef_b && std::memcmp(a->passes, b->passes, sizeof(a->passes)) == 0;
+           a->ef_b == b->ef_b && a->diag == b->diag &&
+           std::memcmp(a->passes, b->passes, sizeof(a->passes)) == 0;
 }
 
 // Per-matrix scratch carving (byte offsets).  gram, linv and the tensor engine's first entries
@@ -114,15 +117,17 @@ Batching make_batches(const orthdion_t* hs, int32_t count) {
     return out;
 }
 
-// Workspace: [status words][P_0 R_0][P_1 R_1]...[scratch of the largest group]
+// Workspace: [status words][diagnostic records][P_0 R_0][P_1 R_1]...[scratch of the largest group]
 struct Layout {
     std::vector<size_t> p_off, r_off;
-    size_t status_off = 0, scratch_off = 0, total = 0;
+    size_t status_off = 0, diag_off = 0, scratch_off = 0, total = 0;
 };
 
 Layout make_layout(const orthdion_t* hs, int32_t count, size_t scratch_bytes) {
     Layout l;
     size_t off = align_up((size_t)count * 4, 256);
+    l.diag_off = off;
+    off += align_up((size_t)count * DIAG_STRIDE * 4, 256);
     l.p_off.resize(count);
     l.r_off.resize(count);
     for (int i = 0; i < count; ++i) {
@@ -277,8 +282,51 @@ void qr_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int
     }
 }
 
+// Diagnostics of one class, after its step: Q^T Q from the engine's Gram product, column
+// statistics of R, optionally the norms of M' and G, then one CTA per matrix for the rest.
+void diag_stage(ClassRun& c, DiagBase db, cudaStream_t st) {
+    const orthdion_plan* p = c.p;
+    const Batch& b = *c.b;
+    const int r = p->r;
+    const Sel gram = sel(W_SCRATCH, c.sc.gram);
+    const int64_t stats_off = c.sc.linv;          // 2 r floats of the (now free) inverse slot
+    {
+        prof::Scope scope(prof::S_DIAG, st);
+        diag_init_kernel<<<(b.count * DIAG_STRIDE + 255) / 256, 256, 0, st>>>(b, db);
+    }
+    if (c.tensor()) {
+        tensor_gram(r, p->passes[1], b, c.sc.ts.q, p->n, gram, 0, st);
+    } else {
+        const Sel sQ = sel(W_Q);
+        launch_simt(b, r, r, p->n, RdPlain{sQ, 1, r}, RdPlain{sQ, 1, r}, EpStore{gram, gram, 0, 1, r, 0},
+                    prof::S_GRAM, st);
+    }
+    {
+        prof::Scope scope(prof::S_DIAG, st);
+        if (r % 4 == 0) {
+            dim3 grid((unsigned)((r + 127) / 128), 1, (unsigned)b.count);
+            diag_colstats4_kernel<<<grid, 1024, 0, st>>>(b, p->n, r, stats_off);
+        } else {
+            dim3 grid((unsigned)((r + 31) / 32), 1, (unsigned)b.count);
+            diag_colstats_kernel<<<grid, 1024, 0, st>>>(b, p->n, r, stats_off);
+        }
+    }
+    if (p->diag & 2) {
+        const int64_t elems = p->m * p->n;
+        const int64_t want = (elems / 4 + 256 * 32 - 1) / (256 * 32);
+        dim3 grid((unsigned)std::max<int64_t>(1, std::min<int64_t>(want, 1184 / std::max(1, b.count) + 1)), 1,
+                  (unsigned)b.count);
+        prof::Scope scope(prof::S_DIAG, st);
+        diag_frob_kernel<<<grid, 256, 0, st>>>(b, elems, p->g_dtype == ORTHDION_DTYPE_BF16, db);
+    }
+    {
+        prof::Scope scope(prof::S_DIAG, st);
+        diag_final_kernel<<<b.count, DIAG_THREADS, 0, st>>>(b, r, c.sc.gram, stats_off, p->diag, p->ef_a, p->ef_b, db);
+    }
+}
+
 // One step of every class of a group, stage by stage.
-void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
+void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, cudaStream_t st) {
     const Sel sP = sel(W_P), sR = sel(W_R), sQ = sel(W_Q);
     std::vector<int> all, orth;
     for (size_t i = 0; i < cls.size(); ++i) {
@@ -335,6 +383,8 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, cudaStream_t st) {
                         EpWeights{cc, dd, p->n, xb}, prof::S_K5, st);
         }
     }
+    for (ClassRun& c : cls)
+        if (c.p->diag) diag_stage(c, db, st);
 }
 
 int check_ptr(const void* p) {
@@ -364,6 +414,7 @@ int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r, float mu, 
     p->x_dtype = ORTHDION_DTYPE_BF16; p->g_dtype = ORTHDION_DTYPE_BF16;
     p->engine = tensor_engine_supports(m, n, r) ? ORTHDION_ENGINE_TENSOR : ORTHDION_ENGINE_SIMT;
     p->passes[0] = 3; p->passes[1] = 3; p->passes[2] = 1; p->passes[3] = 1;
+    p->diag = 0;
     *out = p;
     return ORTHDION_OK;
 }
@@ -426,6 +477,13 @@ int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes) {
     return ORTHDION_OK;
 }
 
+int orthdion_set_diagnostics(orthdion_t h, int32_t mask) {
+    if (!valid(h) || mask < 0 || mask > 3) return ORTHDION_ERR_INVALID_ARG;
+    if (mask == 2) mask = 3;      // the buffer norms are reported together with the factor diagnostics
+    h->diag = mask;
+    return ORTHDION_OK;
+}
+
 size_t orthdion_workspace_bytes_grouped(const orthdion_t* hs, int32_t count) {
     if (!hs || count < 1) return 0;
     for (int i = 0; i < count; ++i)
@@ -480,7 +538,9 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
             cls.push_back(c);
         }
         engine_error() = 0;
-        run_group(cls, merged, st);
+        const DiagBase db{reinterpret_cast<const int32_t*>(ws + lay.status_off),
+                          reinterpret_cast<float*>(ws + lay.diag_off)};
+        run_group(cls, merged, db, st);
         if (engine_error()) {
             std::fprintf(stderr, "orthdion: tensor map setup failed (%d)\n", engine_error());
             rc = ORTHDION_ERR_CUDA;
@@ -579,6 +639,23 @@ int orthdion_last_status(const orthdion_t* hs, int32_t count, void* workspace, v
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     CU_CHECK(cudaMemcpyAsync(flags, workspace, (size_t)count * 4, cudaMemcpyDeviceToHost, st));
     CU_CHECK(cudaStreamSynchronize(st));
+    return ORTHDION_OK;
+}
+
+int orthdion_last_diagnostics(const orthdion_t* hs, int32_t count, void* workspace, void* stream, float* out) {
+    if (!hs || !workspace || !out) return ORTHDION_ERR_NULL;
+    if (count < 1) return ORTHDION_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i)
+        if (!valid(hs[i])) return ORTHDION_ERR_INVALID_ARG;
+    Layout lay = make_layout(hs, count, 0);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const char* ws = reinterpret_cast<const char*>(workspace);
+    CU_CHECK(cudaMemcpy2DAsync(out, ORTHDION_DIAG_FLOATS * 4, ws + lay.diag_off, DIAG_STRIDE * 4,
+                               ORTHDION_DIAG_FLOATS * 4, (size_t)count, cudaMemcpyDeviceToHost, st));
+    CU_CHECK(cudaStreamSynchronize(st));
+    for (int i = 0; i < count; ++i)
+        if (!hs[i]->diag)
+            for (int k = 0; k < ORTHDION_DIAG_FLOATS; ++k) out[(size_t)i * ORTHDION_DIAG_FLOATS + k] = 0.f;
     return ORTHDION_OK;
 }
 

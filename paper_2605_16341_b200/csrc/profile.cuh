@@ -9,11 +9,12 @@
 namespace od {
 namespace prof {
 
-enum Stage : int { S_MISC = 0, S_PACK, S_K1, S_GRAM, S_CHOL, S_APPLY, S_K3, S_COLNORM, S_K5, S_COUNT };
+enum Stage : int { S_MISC = 0, S_PACK, S_K1, S_GRAM, S_CHOL, S_APPLY, S_K3, S_COLNORM, S_K5, S_DIAG, S_COUNT };
 
 inline const char* stage_name(int s) {
     static const char* names[S_COUNT] = {"misc", "pack", "k1_buffer_times_q", "gram", "cholesky_inverse",
-                                         "apply_inverse", "k3_buffer_t_times_p", "colnorm", "k5_feedback_update"};
+                                         "apply_inverse", "k3_buffer_t_times_p", "colnorm", "k5_feedback_update",
+                                         "diagnostics"};
     return (s >= 0 && s < S_COUNT) ? names[s] : "?";
 }
 
