@@ -34,24 +34,27 @@ __global__ void diag_init_kernel(const __grid_constant__ Batch batch, DiagBase d
 }
 
 // Column statistics of R and Q (both n x r fp32, row-major): stats[j] = sum_i R_ij^2,
-// stats[r + j] = sum_i R_ij Q_ij.  One CTA per 32 columns, lanes along columns.
+// stats[r + j] = sum_i R_ij Q_ij, stats[2r + j] = sum_i Q_ij^2.  One CTA per 32 columns, lanes
+// along columns.
 __global__ void __launch_bounds__(1024)
 diag_colstats_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t stats_off) {
     const MatWork& w = batch.w[blockIdx.z];
-    __shared__ float part[2][32][33];
+    __shared__ float part[3][32][33];
     const int lane = threadIdx.x % 32, ry = threadIdx.x / 32;
     const int j = blockIdx.x * 32 + lane;
-    float s = 0.f, t = 0.f;
+    float s = 0.f, t = 0.f, u = 0.f;
     if (j < r)
         for (int64_t i = ry; i < n; i += 32) {
-            const float v = w.R[i * r + j];
+            const float v = w.R[i * r + j], q = w.Q[i * r + j];
             s = fmaf(v, v, s);
-            t = fmaf(v, w.Q[i * r + j], t);
+            t = fmaf(v, q, t);
+            u = fmaf(q, q, u);
         }
     part[0][ry][lane] = s;
     part[1][ry][lane] = t;
+    part[2][ry][lane] = u;
     __syncthreads();
-    if (ry < 2 && j < r) {
+    if (ry < 3 && j < r) {
         float acc = 0.f;
         for (int k = 0; k < 32; ++k) acc += part[ry][k][lane];
         reinterpret_cast<float*>(w.scratch + stats_off)[ry * r + j] = acc;
@@ -62,25 +65,38 @@ diag_colstats_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int6
 __global__ void __launch_bounds__(1024)
 diag_colstats4_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t stats_off) {
     const MatWork& w = batch.w[blockIdx.z];
-    __shared__ __align__(16) float part[2][32][132];
+    __shared__ __align__(16) float part[3][16][132];
     const int lane = threadIdx.x % 32, ry = threadIdx.x / 32;
     const int j = blockIdx.x * 128 + lane * 4;
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f), t = s;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f), t = s, u = s;
     if (j < r)
         for (int64_t i = ry; i < n; i += 32) {
             const float4 a = *reinterpret_cast<const float4*>(w.R + i * r + j);
             const float4 q = *reinterpret_cast<const float4*>(w.Q + i * r + j);
             s.x = fmaf(a.x, a.x, s.x); s.y = fmaf(a.y, a.y, s.y); s.z = fmaf(a.z, a.z, s.z); s.w = fmaf(a.w, a.w, s.w);
             t.x = fmaf(a.x, q.x, t.x); t.y = fmaf(a.y, q.y, t.y); t.z = fmaf(a.z, q.z, t.z); t.w = fmaf(a.w, q.w, t.w);
+            u.x = fmaf(q.x, q.x, u.x); u.y = fmaf(q.y, q.y, u.y); u.z = fmaf(q.z, q.z, u.z); u.w = fmaf(q.w, q.w, u.w);
         }
-    *reinterpret_cast<float4*>(&part[0][ry][lane * 4]) = s;
-    *reinterpret_cast<float4*>(&part[1][ry][lane * 4]) = t;
+    if (ry >= 16) {
+        *reinterpret_cast<float4*>(&part[0][ry - 16][lane * 4]) = s;
+        *reinterpret_cast<float4*>(&part[1][ry - 16][lane * 4]) = t;
+        *reinterpret_cast<float4*>(&part[2][ry - 16][lane * 4]) = u;
+    }
     __syncthreads();
-    if (threadIdx.x < 256) {
+    if (ry < 16) {
+        const float4 s2 = *reinterpret_cast<const float4*>(&part[0][ry][lane * 4]);
+        const float4 t2 = *reinterpret_cast<const float4*>(&part[1][ry][lane * 4]);
+        const float4 u2 = *reinterpret_cast<const float4*>(&part[2][ry][lane * 4]);
+        *reinterpret_cast<float4*>(&part[0][ry][lane * 4]) = make_float4(s.x + s2.x, s.y + s2.y, s.z + s2.z, s.w + s2.w);
+        *reinterpret_cast<float4*>(&part[1][ry][lane * 4]) = make_float4(t.x + t2.x, t.y + t2.y, t.z + t2.z, t.w + t2.w);
+        *reinterpret_cast<float4*>(&part[2][ry][lane * 4]) = make_float4(u.x + u2.x, u.y + u2.y, u.z + u2.z, u.w + u2.w);
+    }
+    __syncthreads();
+    if (threadIdx.x < 384) {
         const int which = threadIdx.x / 128, c = threadIdx.x % 128;
         if (blockIdx.x * 128 + c < r) {
             float acc = 0.f;
-            for (int k = 0; k < 32; ++k) acc += part[which][k][c];
+            for (int k = 0; k < 16; ++k) acc += part[which][k][c];
             reinterpret_cast<float*>(w.scratch + stats_off)[which * r + blockIdx.x * 128 + c] = acc;
         }
     }
@@ -175,7 +191,10 @@ __device__ float diag_tridiag_max(const float* alpha, const float* beta, int k, 
 }
 
 // One CTA per matrix: finishes the diagnostics.  `gram` holds Q^T Q (at least its lower
-// triangle; it is mirrored in place first).  nu^2 is the largest eigenvalue of Q^T Q: Lanczos
+// triangle; it is mirrored in place first).  Its diagonal is replaced by the column squares of Q
+// summed in fp32 registers: the tensor-core accumulation rounds towards zero, which lowers a sum
+// of n positive terms by about 5e-9 n (relative), visible in nu of an orthonormal Q at n ~ 10^4;
+// the off-diagonal entries keep that bias (it enters nu only through nu^2 - 1).  nu^2 is the largest eigenvalue of Q^T Q: Lanczos
 // iteration from a fixed pseudo-random start (no re-orthogonalisation: only the top Ritz value is
 // used, which converges regardless), the top Ritz value taken every fourth step and the iteration
 // stopped once it has moved by less than 1e-6 (relative), the Krylov space is exhausted, or
@@ -196,6 +215,7 @@ diag_final_kernel(const __grid_constant__ Batch batch, int r, int64_t gram_off, 
     float* g = reinterpret_cast<float*>(w.scratch + gram_off);
     const float* colsq = reinterpret_cast<const float*>(w.scratch + stats_off);
     const float* rq = colsq + r;
+    const float* qsq = colsq + 2 * r;
 
     // column norms of R: entropy of their distribution, ||R||_F, <R, Q>
     float s_sum = 0.f, sq_sum = 0.f, rq_sum = 0.f;
@@ -216,6 +236,7 @@ diag_final_kernel(const __grid_constant__ Batch batch, int r, int64_t gram_off, 
     // mirror the lower triangle
     for (int i = warp; i < r; i += DIAG_THREADS / 32)
         for (int j = i + 1 + lane; j < r; j += 32) g[(int64_t)i * r + j] = g[(int64_t)j * r + i];
+    for (int j = tid; j < r; j += DIAG_THREADS) g[(int64_t)j * r + j] = qsq[j];
     float nrm2 = 0.f;
     for (int j = tid; j < r; j += DIAG_THREADS) {
         uint32_t h = (uint32_t)j * 2654435761u + 12345u;

@@ -289,7 +289,7 @@ void diag_stage(ClassRun& c, DiagBase db, cudaStream_t st) {
     const Batch& b = *c.b;
     const int r = p->r;
     const Sel gram = sel(W_SCRATCH, c.sc.gram);
-    const int64_t stats_off = c.sc.linv;          // 2 r floats of the (now free) inverse slot
+    const int64_t stats_off = c.sc.linv;          // 3 r floats of the (now free) inverse slot
     {
         prof::Scope scope(prof::S_DIAG, st);
         diag_init_kernel<<<(b.count * DIAG_STRIDE + 255) / 256, 256, 0, st>>>(b, db);

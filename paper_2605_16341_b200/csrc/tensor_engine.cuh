@@ -1221,17 +1221,18 @@ inline int64_t img_bytes(int64_t rows, int64_t cols, int planes = 2) {
 }
 inline ImgRef no_img() { ImgRef im; im.off = -1; im.rows_pad = 0; im.panels = 0; im.planes = 0; im.pad = 0; return im; }
 
-// The offsets of linv and colsq depend on r only, so that one Cholesky launch can serve
-// matrices of different shapes.
+// The offsets of linv, cnorm, rscale and colsq depend on r only (everything whose size depends on
+// the matrix shape comes after them), so that one Cholesky launch can serve matrices of
+// different shapes.
 // half_planes: P, R, Q carry the fp16 plane (fused pass in fp16).
 inline size_t tensor_scratch_layout(int64_t m, int64_t n, int32_t r, bool half_planes, size_t off, TensorScratch* ts) {
     const int64_t kmax = std::max(m, n);
     off = (off + 1023) / 1024 * 1024;
     auto take = [&](int64_t bytes) { int64_t o = (int64_t)off; off += (size_t)((bytes + 1023) / 1024 * 1024); return o; };
     ts->linv = make_img(take(img_bytes(r, r)), r, r);
-    ts->colsq = take(4 * ((kmax + 127) / 128) * (int64_t)r * 4);
     ts->cnorm = take((int64_t)r * 4);
     ts->rscale = take(16);
+    ts->colsq = take(4 * ((kmax + 127) / 128) * (int64_t)r * 4);
     const int pl = half_planes ? 3 : 2;
     ts->qprev = make_img(take(img_bytes(n, r)), n, r);
     ts->w0 = make_img(take(img_bytes(kmax, r)), kmax, r);

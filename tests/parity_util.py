@@ -14,6 +14,15 @@ TOL_CHAIN = 1e-3      # the same after 10 chained steps
 TOL_ORTHO = 1e-5      # max |Q^T Q - I|
 
 
+def poisoned_workspace(nbytes: int) -> torch.Tensor:
+    """A workspace whose every byte is 0x7f (floats of 3.4e38, bf16/fp16 values far out of range):
+    the step must not depend on what the workspace held before, and anything it reads without
+    having written it first shows up as a wrong result instead of passing on zeroed memory."""
+    ws = od.alloc_workspace(nbytes)
+    ws.fill_(0x7F)
+    return ws
+
+
 def f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().double().cpu().numpy()
 
@@ -39,7 +48,7 @@ class GpuMatrix:
         for k, v in (passes or {}).items():
             od.orthdion_set_passes(self.h, k, v)
         self.X, self.M, self.Q = X.cuda().contiguous(), M.cuda().contiguous(), Q.cuda().contiguous()
-        self.ws = od.alloc_workspace(od.orthdion_workspace_bytes(self.h))
+        self.ws = poisoned_workspace(od.orthdion_workspace_bytes(self.h))
         self.eta, self.wd, self.scale = eta, wd, 1.0 if scale is None else scale
 
     def step(self, G):

@@ -16,7 +16,7 @@ from oracle import orthdion_oracle as orc
 from paper_2605_16341_b200 import binding as od
 from paper_2605_16341_b200 import workloads as wl
 
-from parity_util import GpuMatrix, f64, oracle_mode
+from parity_util import GpuMatrix, f64, oracle_mode, poisoned_workspace
 
 pytestmark = pytest.mark.gpu
 
@@ -126,7 +126,7 @@ def test_diagnostics_do_not_change_the_step_and_index_by_matrix():
             hs.append(h)
             Xs.append(X.cuda().clone()); Ms.append(M.cuda().clone())
             Gs.append(G.cuda().clone()); Qs.append(Q.cuda().clone())
-        ws = od.alloc_workspace(od.orthdion_workspace_bytes_grouped(hs))
+        ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
         od.orthdion_step_grouped(od.PointerTable(hs, Xs, Ms, Gs, Qs), ws)
         torch.cuda.synchronize()
         assert all(s == 0 for s in od.orthdion_last_status(hs, ws))
@@ -165,3 +165,53 @@ def test_set_diagnostics_rejects_bad_masks():
         with pytest.raises(od.OrthDionError):
             od.orthdion_set_diagnostics(h, bad)
     od.orthdion_destroy(h)
+
+
+@pytest.mark.parametrize("mode", [od.MODE_ORTH, od.MODE_COLNORM], ids=["orth", "colnorm"])
+def test_diagnostics_at_full_size_in_the_grouped_launch(mode):
+    """One layer of the 8B workload (r = 512, n up to 14336) in the benchmark's launch
+    configuration.  Every matrix: against float64 library routines applied to the device's own
+    state (matrix 2-norm of Q, column norms of R, Frobenius norms).  The 1024 x 4096 matrix also
+    against the oracle's own step."""
+    w = wl.workload("cfg4", layers=1)
+    dev = torch.device("cuda")
+    plan, hs, M0s, Gs, Xs, Ms, Qs, Q0s, X0s = {}, [], [], [], [], [], [], [], []
+    for i, spec in enumerate(w.matrices):
+        key = (spec.m, spec.n, spec.r)
+        if key not in plan:
+            plan[key] = od.orthdion_create(spec.m, spec.n, spec.r, w.mu, w.eta, w.wd, mode)
+            od.orthdion_set_diagnostics(plan[key], 3)
+        hs.append(plan[key])
+        X, M, Q = wl.initial_state(spec, 0, i, device=dev)
+        M = 0.02 * torch.randn(spec.m, spec.n, device=dev, generator=torch.Generator(device=dev).manual_seed(50 + i))
+        G = wl.gradient(w, spec, 0, i, 0, wl.grad_basis(w, spec, 0, i, device=dev), device=dev)
+        X0s.append(X.clone()); M0s.append(M.clone()); Q0s.append(Q.clone()); Gs.append(G)
+        Xs.append(X); Ms.append(M); Qs.append(Q)
+    ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
+    od.orthdion_step_grouped(od.PointerTable(hs, Xs, Ms, Gs, Qs), ws)
+    torch.cuda.synchronize()
+    assert od.orthdion_last_status(hs, ws) == [0] * len(hs)
+    diags = od.orthdion_last_diagnostics(hs, ws)
+    by_oracle = 0
+    for i, spec in enumerate(w.matrices):
+        d = diags[i]
+        P, R = od.orthdion_get_factors(hs, i, ws, (spec.m, spec.n, spec.r))
+        Rd, Qd = R.double(), Qs[i].double()
+        s = Rd.norm(dim=0)
+        p = s / s.sum()
+        want = dict(nu=float(torch.linalg.matrix_norm(Qd, ord=2)),
+                    erank=float(torch.exp(-(p * torch.log(p)).sum())),
+                    tr_t2=float((Rd * Qd).sum()), norm_r=float(Rd.norm()),
+                    norm_m=float(Ms[i].double().norm()), norm_g=float(Gs[i].double().norm()),
+                    norm_b=float((M0s[i].double() + Gs[i].double()).norm()))
+        compare(d, want, 3)
+        if mode == od.MODE_ORTH:
+            assert abs(d["nu"] - 1.0) <= 1e-5
+        if spec.name == "l0.k":
+            ref = orc.step(f64(X0s[i]), f64(M0s[i]), f64(Gs[i]), f64(Q0s[i]), eta=w.eta, mu=w.mu, wd=w.wd,
+                           mode=oracle_mode(mode))
+            compare(d, oracle_diagnostics(ref, Gs[i], mode), 3)
+            by_oracle += 1
+    assert by_oracle == 1
+    for h in plan.values():
+        od.orthdion_destroy(h)

@@ -15,7 +15,7 @@ from oracle import orthdion_oracle as orc
 from paper_2605_16341_b200 import binding as od
 from paper_2605_16341_b200 import workloads as wl
 
-from parity_util import TOL_ORTHO, TOL_STEP, f64, rel
+from parity_util import TOL_ORTHO, TOL_STEP, f64, poisoned_workspace, rel
 
 pytestmark = pytest.mark.gpu
 
@@ -71,7 +71,7 @@ def test_one_layer_of_the_grouped_workloads(cfg, mode):
         G = wl.gradient(w, spec, 0, i, 0, basis, device=dev)
         X0s.append(X.clone()); M0s.append(M.clone()); Q0s.append(Q.clone()); Gs.append(G)
         Xs.append(X); Ms.append(M); Qs.append(Q)
-    ws = od.alloc_workspace(od.orthdion_workspace_bytes_grouped(hs))
+    ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
     table = od.PointerTable(hs, Xs, Ms, Gs, Qs)
     od.orthdion_step_grouped(table, ws)
     torch.cuda.synchronize()
@@ -113,7 +113,7 @@ def test_rank_sweep_ends_on_the_mlp_matrix(r, mode):
     G = wl.gradient(w, spec, 0, 0, 0, basis, device=dev)
     X0, M0, Q0 = X.clone(), M.clone(), Q.clone()
     h = od.orthdion_create(spec.m, spec.n, spec.r, w.mu, w.eta, w.wd, mode)
-    ws = od.alloc_workspace(od.orthdion_workspace_bytes(h))
+    ws = poisoned_workspace(od.orthdion_workspace_bytes(h))
     od.orthdion_step(h, X, M, G, Q, ws)
     torch.cuda.synchronize()
     assert od.orthdion_last_status([h], ws) == [0]

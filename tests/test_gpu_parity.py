@@ -13,7 +13,7 @@ from paper_2605_16341_b200 import binding as od
 from paper_2605_16341_b200 import workloads as wl
 
 from parity_util import (TOL_CHAIN, TOL_ORTHO, TOL_STEP, GpuMatrix, check_bf16_rounding,
-                         delta_x_from_factors, f64, oracle_mode, rel)
+                         delta_x_from_factors, f64, oracle_mode, poisoned_workspace, rel)
 
 pytestmark = pytest.mark.gpu
 
@@ -217,7 +217,7 @@ def test_grouped_matches_single_and_is_deterministic(engine):
         hs.append(h)
     dev = [tuple(t.cuda() for t in s) for s in st]
     Gd = [g.cuda() for g in Gs]
-    ws = od.alloc_workspace(od.orthdion_workspace_bytes_grouped(hs))
+    ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
     table = od.PointerTable(hs, [d[0] for d in dev], [d[1] for d in dev], Gd, [d[2] for d in dev])
     for _ in range(2):
         od.orthdion_step_grouped(table, ws)
