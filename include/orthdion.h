@@ -175,6 +175,28 @@ int orthdion_set_diagnostics(orthdion_t h, int32_t mask);
 int orthdion_last_diagnostics(const orthdion_t* hs, int32_t count, void* workspace, void* stream,
                               float* out);
 
+/* Adaptive rank (appendix algorithm "Ada-Orth-Dion Rank Selection").  The estimate e_t is slot [1]
+ * of the diagnostics (effective rank from the column norms of R).  Host arithmetic in double:
+ *     ema    = alpha * e_t + (1 - alpha) * ema_prev
+ *     target = ceil(gamma * ema)
+ *     r_next = clip(target, r_min, r_max) rounded to the nearest multiple of `multiple` (tie: up)
+ * r_min and r_max must be positive multiples of `multiple` (the paper rounds to 8; the TENSOR
+ * engine needs 16), 0 <= alpha <= 1, gamma > 0 (the paper's text has 1.1, its table 1.425).  The
+ * paper does not say how the average starts: pass ema_prev = e_t on the first step.  r_t is the
+ * current rank (the rule is stated with it; the caller resizes when *r_next differs). */
+int orthdion_rank_policy(double e_t, int32_t r_t, double ema_prev, int32_t r_min, int32_t r_max,
+                         double alpha, double gamma, int32_t multiple, double* ema_out, int32_t* r_next);
+
+/* "Resize U, V to rank r_{t+1} (truncate or pad)" for the one factor that is carried between
+ * steps: Q_new (n x r_new, device, row-major) receives the leading min(r_old, r_new) columns of
+ * Q_old (n x r_old) and, when r_new > r_old, the columns of `pad` (n x (r_new - r_old), device,
+ * row-major; may be null otherwise).  The paper does not say what the new columns hold: the caller
+ * supplies them (any columns that keep B*Q of full column rank serve the power iteration, e.g.
+ * N(0, 1/n) entries).  Q_new must not alias Q_old.  Enqueued on `stream`; the next step then uses
+ * a plan created with r_new (plans of different rank are packed separately by the grouped step). */
+int orthdion_resize_factor(const float* Q_old, int64_t n, int32_t r_old, float* Q_new, int32_t r_new,
+                           const float* pad, void* stream);
+
 /* Number of kernels this library has launched so far in this process (monotonic). */
 int64_t orthdion_launch_count(void);
 

@@ -209,6 +209,44 @@ def effective_rank_estimate(R):
 
 
 # ----------------------------------------------------------------------------------
+# Ada-Orth-Dion rank selection (appendix algorithm "Ada-Orth-Dion Rank Selection")
+# ----------------------------------------------------------------------------------
+def rank_policy(e_t, r_t, ema_prev, r_min, r_max, alpha, gamma, multiple=8):
+    """One application of the rank-selection rule.  Returns (ema_t, r_next).
+
+        ema_t    = alpha * e_t + (1 - alpha) * ema_prev
+        r_target = ceil(gamma * ema_t)
+        r_next   = clip(r_target, r_min, r_max), rounded to a multiple of `multiple`
+
+    Readings where the paper is silent: "rounded" is to the nearest multiple, a tie going up;
+    r_min and r_max are multiples of `multiple` themselves, so rounding cannot leave the bounds;
+    all arithmetic in float64.  r_t is carried only because the rule is stated with it (the
+    resize happens when r_next != r_t)."""
+    if r_min % multiple or r_max % multiple or r_min < multiple or r_max < r_min:
+        raise ValueError("bounds must be positive multiples of `multiple`")
+    ema_t = float(alpha) * float(e_t) + (1.0 - float(alpha)) * float(ema_prev)
+    r_target = int(np.ceil(float(gamma) * ema_t))
+    clipped = min(max(r_target, r_min), r_max)
+    r_next = int(np.floor(clipped / multiple + 0.5)) * multiple
+    return ema_t, r_next
+
+
+def resize_factor(Q, r_new, pad=None):
+    """Resize the warm-start factor to r_new columns: keep the leading columns (truncate), or
+    append the given columns (pad).  The paper only says "truncate or pad"; the reading taken is
+    that the new columns are supplied by the caller (any columns that keep B Q of full rank will
+    do for the power iteration; the tests draw them N(0, 1/n))."""
+    Q = np.asarray(Q, dtype=np.float64)
+    n, r = Q.shape
+    if r_new <= r:
+        return Q[:, :r_new].copy()
+    pad = np.asarray(pad, dtype=np.float64)
+    if pad.shape != (n, r_new - r):
+        raise ValueError("pad must be n x (r_new - r)")
+    return np.concatenate([Q, pad], axis=1)
+
+
+# ----------------------------------------------------------------------------------
 # Storage rounding (bf16 round-to-nearest-even), for comparing stored weights
 # ----------------------------------------------------------------------------------
 def round_to_bf16(x):

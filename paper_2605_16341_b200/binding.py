@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
     L.orthdion_last_status.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(i32)]
     L.orthdion_set_diagnostics.argtypes = [vp, i32]
     L.orthdion_last_diagnostics.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(ctypes.c_float)]
+    dbl = ctypes.c_double
+    L.orthdion_rank_policy.argtypes = [dbl, i32, dbl, i32, i32, dbl, dbl, i32, ctypes.POINTER(dbl),
+                                       ctypes.POINTER(i32)]
+    L.orthdion_resize_factor.argtypes = [vp, i64, i32, vp, i32, vp, vp]
     L.orthdion_version.restype = ctypes.c_char_p
     L.orthdion_launch_count.restype = i64
     L.orthdion_profile_begin.argtypes = [i32]
@@ -90,7 +94,7 @@ def lib() -> ctypes.CDLL:
     L.orthdion_stage_name.restype = ctypes.c_char_p
     for name in ("create", "destroy", "set_dtypes", "set_lr", "set_scale", "set_ef", "set_engine",
                  "set_passes", "step", "step_grouped", "step_noalloc", "get_factors", "last_status",
-                 "set_diagnostics", "last_diagnostics"):
+                 "set_diagnostics", "last_diagnostics", "rank_policy", "resize_factor"):
         getattr(L, "orthdion_" + name).restype = i32
     _lib = L
     return L
@@ -100,7 +104,8 @@ EXPORTED = ["orthdion_create", "orthdion_destroy", "orthdion_set_dtypes", "orthd
             "orthdion_set_scale", "orthdion_set_ef", "orthdion_set_engine", "orthdion_set_passes",
             "orthdion_workspace_bytes", "orthdion_workspace_bytes_grouped", "orthdion_step",
             "orthdion_step_grouped", "orthdion_step_noalloc", "orthdion_get_factors", "orthdion_last_status",
-            "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_version",
+            "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_rank_policy",
+            "orthdion_resize_factor", "orthdion_version",
             "orthdion_launch_count", "orthdion_profile_begin", "orthdion_profile_end", "orthdion_stage_count",
             "orthdion_stage_name"]
 
@@ -259,6 +264,23 @@ def orthdion_last_diagnostics(hs, workspace, stream=None):
     _check(lib().orthdion_last_diagnostics(_harr(hs), len(hs), _dev_ptr(workspace, "workspace"),
                                            _stream_ptr(stream), out), "orthdion_last_diagnostics")
     return [dict(zip(DIAG_NAMES, out[i * DIAG_FLOATS:(i + 1) * DIAG_FLOATS])) for i in range(len(hs))]
+
+
+def orthdion_rank_policy(e_t, r_t, ema_prev, r_min, r_max, alpha, gamma, multiple=8):
+    """Returns (ema_t, r_next) of the rank-selection rule (host arithmetic inside the library)."""
+    ema, r_next = ctypes.c_double(), ctypes.c_int32()
+    _check(lib().orthdion_rank_policy(e_t, r_t, ema_prev, r_min, r_max, alpha, gamma, multiple,
+                                      ctypes.byref(ema), ctypes.byref(r_next)), "orthdion_rank_policy")
+    return ema.value, r_next.value
+
+
+def orthdion_resize_factor(Q_old, Q_new, pad=None, stream=None):
+    n, r_old = Q_old.shape
+    r_new = Q_new.shape[1]
+    assert Q_new.shape[0] == n and Q_old.dtype == Q_new.dtype == torch.float32
+    _check(lib().orthdion_resize_factor(_dev_ptr(Q_old, "Q_old"), n, r_old, _dev_ptr(Q_new, "Q_new"), r_new,
+                                        _dev_ptr(pad, "pad") if pad is not None else None,
+                                        _stream_ptr(stream)), "orthdion_resize_factor")
 
 
 def orthdion_launch_count() -> int:

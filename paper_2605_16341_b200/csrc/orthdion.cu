@@ -3,6 +3,7 @@
 #include "../../include/orthdion.h"
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -13,6 +14,7 @@
 #include "factor_kernels.cuh"
 #include "factor_tc.cuh"
 #include "diag_kernels.cuh"
+#include "rank_kernels.cuh"
 #include "simt_kernels.cuh"
 #include "tensor_engine.cuh"
 
@@ -656,6 +658,48 @@ int orthdion_last_diagnostics(const orthdion_t* hs, int32_t count, void* workspa
     for (int i = 0; i < count; ++i)
         if (!hs[i]->diag)
             for (int k = 0; k < ORTHDION_DIAG_FLOATS; ++k) out[(size_t)i * ORTHDION_DIAG_FLOATS + k] = 0.f;
+    return ORTHDION_OK;
+}
+
+int orthdion_rank_policy(double e_t, int32_t r_t, double ema_prev, int32_t r_min, int32_t r_max, double alpha,
+                         double gamma, int32_t multiple, double* ema_out, int32_t* r_next) {
+    (void)r_t;   // part of the rule's statement; the caller resizes when *r_next differs from it
+    if (!ema_out || !r_next) return ORTHDION_ERR_NULL;
+    if (multiple < 1 || r_min < multiple || r_max < r_min || r_min % multiple || r_max % multiple)
+        return ORTHDION_ERR_INVALID_ARG;
+    if (!(e_t == e_t) || !(ema_prev == ema_prev) || !(alpha >= 0.0 && alpha <= 1.0) || !(gamma > 0.0))
+        return ORTHDION_ERR_INVALID_ARG;
+    const double ema = alpha * e_t + (1.0 - alpha) * ema_prev;
+    double target = std::ceil(gamma * ema);
+    if (!(target >= (double)r_min)) target = (double)r_min;
+    if (target > (double)r_max) target = (double)r_max;
+    *ema_out = ema;
+    *r_next = (int32_t)std::floor(target / multiple + 0.5) * multiple;
+    return ORTHDION_OK;
+}
+
+int orthdion_resize_factor(const float* Q_old, int64_t n, int32_t r_old, float* Q_new, int32_t r_new,
+                           const float* pad, void* stream) {
+    if (!Q_old || !Q_new) return ORTHDION_ERR_NULL;
+    if (n < 1 || n > (1 << 24) || r_old < 1 || r_new < 1 || r_old > kMaxRank || r_new > kMaxRank)
+        return ORTHDION_ERR_INVALID_ARG;
+    if (r_new > r_old && !pad) return ORTHDION_ERR_NULL;
+    if (Q_old == Q_new) return ORTHDION_ERR_INVALID_ARG;
+    int e;
+    if ((e = check_ptr(Q_old)) || (e = check_ptr(Q_new)) || (r_new > r_old && (e = check_ptr(pad)))) return e;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int padw = r_new > r_old ? r_new - r_old : 0;
+    const bool vec = r_old % 4 == 0 && r_new % 4 == 0 && padw % 4 == 0;
+    const int64_t total = n * (vec ? r_new / 4 : r_new);
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, 148 * 16));
+    prof::Scope scope(prof::S_MISC, st);
+    if (vec) resize_factor_kernel<4><<<grid, 256, 0, st>>>(Q_old, n, r_old, Q_new, r_new, pad);
+    else resize_factor_kernel<1><<<grid, 256, 0, st>>>(Q_old, n, r_old, Q_new, r_new, pad);
+    cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) {
+        std::fprintf(stderr, "orthdion: launch failed: %s\n", cudaGetErrorString(ce));
+        return ORTHDION_ERR_CUDA;
+    }
     return ORTHDION_OK;
 }
 

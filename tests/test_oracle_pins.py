@@ -335,3 +335,55 @@ def test_effective_rank_estimate_extremes():
     assert abs(orc.effective_rank_estimate(np.eye(6)) - 6.0) < 1e-12       # flat spectrum
     R = np.zeros((5, 4)); R[:, 0] = 1.0; R[:, 1:] = 1e-300
     assert abs(orc.effective_rank_estimate(R) - 1.0) < 1e-9                  # one dominant column
+
+
+# ------------------------------------------------------------------ rank selection (Ada-Orth-Dion)
+def test_rank_policy_worked_examples():
+    # alpha = 1: no memory; gamma = 1: the target is the estimate itself, rounded up to an integer
+    assert orc.rank_policy(40.0, 64, 123.0, 8, 512, 1.0, 1.0) == (40.0, 40)
+    assert orc.rank_policy(40.2, 64, 0.0, 8, 512, 1.0, 1.0) == (40.2, 40)        # ceil 41 -> nearest multiple 40
+    assert orc.rank_policy(43.5, 64, 0.0, 8, 512, 1.0, 1.0)[1] == 48             # ceil 44: tie goes up
+    assert orc.rank_policy(44.5, 64, 0.0, 8, 512, 1.0, 1.0)[1] == 48             # ceil 45 -> 48
+    # EMA by hand: 0.25 * 100 + 0.75 * 60 = 70; gamma 1.5 -> 105 -> 104
+    ema, r = orc.rank_policy(100.0, 64, 60.0, 8, 512, 0.25, 1.5)
+    assert ema == 70.0 and r == 104
+    # clipping at both ends, with bounds that are multiples of 16
+    assert orc.rank_policy(3.0, 64, 3.0, 16, 256, 0.5, 1.1, multiple=16)[1] == 16
+    assert orc.rank_policy(900.0, 64, 900.0, 16, 256, 0.5, 1.1, multiple=16)[1] == 256
+    # alpha = 0 keeps the old average whatever the new estimate says
+    assert orc.rank_policy(500.0, 64, 32.0, 8, 512, 0.0, 1.0) == (32.0, 32)
+    with pytest.raises(ValueError):
+        orc.rank_policy(10.0, 64, 10.0, 12, 512, 0.5, 1.1)                        # bound not a multiple of 8
+
+
+def test_rank_policy_is_monotone_and_stays_in_bounds():
+    g = np.random.default_rng(3)
+    for _ in range(200):
+        e, prev = g.uniform(1, 600, 2)
+        alpha, gamma = g.uniform(0, 1), g.uniform(0.8, 1.6)
+        ema, r = orc.rank_policy(e, 64, prev, 16, 512, alpha, gamma)
+        assert min(e, prev) - 1e-9 <= ema <= max(e, prev) + 1e-9
+        assert 16 <= r <= 512 and r % 8 == 0
+        assert abs(r - min(max(np.ceil(gamma * ema), 16), 512)) <= 4              # nearest multiple of 8
+        assert orc.rank_policy(e + 50, 64, prev, 16, 512, alpha, gamma)[1] >= r    # monotone in the estimate
+
+
+def test_effective_rank_estimate_of_k_equal_columns_is_k():
+    R = np.zeros((7, 10))
+    R[:, :4] = np.random.default_rng(0).standard_normal((7, 4))
+    R[:, :4] /= np.linalg.norm(R[:, :4], axis=0)
+    assert abs(orc.effective_rank_estimate(3.0 * R) - 4.0) < 1e-12                # scale-free, counts equal columns
+    R[:, 1] *= 2.0                                                                # p = (1/5, 2/5, 1/5, 1/5)
+    want = np.exp(-(3 * 0.2 * np.log(0.2) + 0.4 * np.log(0.4)))
+    assert abs(orc.effective_rank_estimate(R) - want) < 1e-12
+
+
+def test_resize_factor_truncates_and_pads():
+    Q = np.arange(12.0).reshape(4, 3)
+    assert np.array_equal(orc.resize_factor(Q, 2), Q[:, :2])
+    assert np.array_equal(orc.resize_factor(Q, 3), Q)
+    pad = -np.ones((4, 2))
+    out = orc.resize_factor(Q, 5, pad)
+    assert out.shape == (4, 5) and np.array_equal(out[:, :3], Q) and np.array_equal(out[:, 3:], pad)
+    with pytest.raises(ValueError):
+        orc.resize_factor(Q, 5, np.ones((4, 1)))
