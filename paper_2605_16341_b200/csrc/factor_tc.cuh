@@ -17,6 +17,8 @@
 //   trailing update  W22 -= L21 L21^T, lower tiles only                (tile products, depth 32)
 // then the inverse of the factor by combining diagonal blocks pairwise (32, 64, 128, ...):
 //   inv [[A, 0], [B, C]] = [[Ai, 0], [-Ci B Ai, Ci]]                   (tile products)
+// The later passes of a CholeskyQR see a Gram matrix I + E with E tiny; when a rigorous bound on
+// |E|_2 is small enough, L^{-1} = I - Phi(E) (first order) replaces the factorisation.
 #pragma once
 #include "common.cuh"
 #include "factor_kernels.cuh"
@@ -28,6 +30,7 @@ constexpr int CT_NB = 32;
 constexpr int CT_KC = 32;             // depth of one staged chunk
 constexpr int CT_LDK = 40;            // staged rows: 32 bf16 + 8 of padding (conflict-free fragment loads)
 constexpr int CT_MAX_TASKS = 160;
+constexpr float CT_SERIES_LIMIT = 1.4e-3f;   // bound on |Gram - I|_2 below which L^{-1} = I - Phi(E) is used
 
 // C(i,j) = beta*C(i,j) + alpha * sum_{k in [kbeg,kend)} A(i,k) B(k,j), i < Mt <= 64, j < Nt <= 64.
 // A(i,k) = A[i*a_rs + k];  B(k,j) = B[k*b_rs + j*b_cs] with b_rs == 1 (k contiguous) or b_cs == 1.
@@ -226,6 +229,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     __shared__ __align__(16) __nv_bfloat16 s_stage[4 * 64 * CT_LDK];
     __shared__ TcTask s_tasks[CT_MAX_TASKS];
     __shared__ float s_diag[1024];
+    __shared__ float s_rowsum[1024];
     __shared__ float red[8];
     __shared__ int s_ntasks, s_fail, s_status;
     __shared__ float s_trace, s_dmin, s_dmax;
@@ -276,6 +280,62 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         return;
     }
 
+    // ---- later passes of the QR: the Gram matrix is I + E with E small ------------------------
+    // L = I + X with X + X^T + X X^T = E, so L^{-1} = I - Phi(E) + O(|E|^2), Phi = strict lower part
+    // plus half the diagonal.  |E|_2 <= max row sum of |E| (E is symmetric); when that bound is
+    // below CT_SERIES_LIMIT the dropped terms are below 2e-6 and the factorisation is skipped.
+    bool series = false;
+    if (a.pass >= 2) {
+        float colacc[32];
+#pragma unroll
+        for (int t = 0; t < 32; ++t) colacc[t] = 0.f;
+        for (int i = tid; i < r; i += CT_THREADS) s_rowsum[i] = fabsf(s_diag[i] - 1.f);
+        __syncthreads();
+        for (int i = warp; i < r; i += CT_THREADS / 32) {
+            float rs = 0.f;
+#pragma unroll
+            for (int t = 0; t < 32; ++t) {
+                const int j = lane + 32 * t;
+                if (j < i) {
+                    const float v = fabsf(A[i * r + j]);
+                    rs += v; colacc[t] += v;
+                }
+            }
+            for (int o = 16; o; o >>= 1) rs += __shfl_xor_sync(0xffffffffu, rs, o);
+            if (lane == 0) atomicAdd(&s_rowsum[i], rs);
+        }
+#pragma unroll
+        for (int t = 0; t < 32; ++t)
+            if (lane + 32 * t < r && colacc[t] != 0.f) atomicAdd(&s_rowsum[lane + 32 * t], colacc[t]);
+        __syncthreads();
+        float mx = 0.f;
+        for (int i = tid; i < r; i += CT_THREADS) mx = fmaxf(mx, s_rowsum[i]);
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) red[warp] = mx;
+        __syncthreads();
+        mx = 0.f;
+        for (int i = 0; i < CT_THREADS / 32; ++i) mx = fmaxf(mx, red[i]);
+        series = mx <= CT_SERIES_LIMIT;          // false for NaN
+        __syncthreads();
+    }
+    if (series) {
+        const int r4 = r / 4;
+        for (int q = tid; q < r * r4; q += CT_THREADS) {
+            const int i = q / r4, j4 = (q - i * r4) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (j4 <= i) {
+                const float4 g = *reinterpret_cast<const float4*>(A + i * r + j4);
+                const float dg = 0.5f * (3.f - s_diag[i]);
+                v.x = j4 + 0 < i ? -g.x : (j4 + 0 == i ? dg : 0.f);
+                v.y = j4 + 1 < i ? -g.y : (j4 + 1 == i ? dg : 0.f);
+                v.z = j4 + 2 < i ? -g.z : (j4 + 2 == i ? dg : 0.f);
+                v.w = j4 + 3 < i ? -g.w : (j4 + 3 == i ? dg : 0.f);
+            }
+            *reinterpret_cast<float4*>(W + i * r + j4) = v;
+        }
+        __syncthreads();
+    }
+
     auto add_task = [&](float* C, int c_rs, int c_cs, const float* A_, int a_rs, const float* B_, int b_rs, int b_cs,
                         int Mt, int Nt, int kbeg, int kend, float alpha, float beta, bool lower_only, int rg0, int cg0) {
         TcTask& t = s_tasks[s_ntasks++];
@@ -285,7 +345,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         t.alpha = alpha; t.beta = beta;
     };
 
-    bool ok = false;
+    bool ok = series;
     const int max_attempts = (a.pass == 1) ? 2 : 1;
     for (int attempt = 0; attempt < max_attempts && !ok; ++attempt) {
         const float shift = attempt ? a.shift_rel * trace : 0.f;
@@ -378,7 +438,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     }
 
     // ---- inverse of the lower factor: the diagonal blocks are inverted already; combine pairwise
-    for (int s = CT_NB; s < r; s *= 2) {
+    for (int s = CT_NB; s < r && !series; s *= 2) {
         const int npairs = (r + 2 * s - 1) / (2 * s);
         // step 1: T = B * Ai, kept transposed in the (unused, zero) mirror block above the diagonal
         if (tid == 0) {
