@@ -43,10 +43,13 @@ enum AMode : int { A_IMG_K = 0, A_IMG_MN = 1, A_BUF_ROW = 2, A_BUF_COL = 3 };
 enum NMode : int { N_IMG_K = 0, N_IMG_MN = 1 };
 enum EpiMode : int { EPI_STORE = 0, EPI_K5 = 1 };
 
-__host__ __device__ constexpr int epi_warps(int epi) { return epi == EPI_K5 ? 8 : 4; }
 __host__ __device__ constexpr bool a_is_buf(int amode) { return amode == A_BUF_ROW || amode == A_BUF_COL; }
+// Eight epilogue warps (two per tensor-memory lane quarter, splitting the columns) wherever the
+// epilogue is a large share of a tile's time: the fused pass and the image-to-image products of
+// the QR.  The products that form B have sixteen transform warps already and a short epilogue.
+__host__ __device__ constexpr int epi_warps(int amode, int epi) { return (epi == EPI_K5 || !a_is_buf(amode)) ? 8 : 4; }
 __host__ __device__ constexpr int gemm_threads(int amode, int epi) {
-    return 32 * (2 + epi_warps(epi) + (a_is_buf(amode) ? NUM_XF_WARPS : 0));
+    return 32 * (2 + epi_warps(amode, epi) + (a_is_buf(amode) ? NUM_XF_WARPS : 0));
 }
 
 // Where the result of an EPI_STORE product goes.
@@ -371,7 +374,7 @@ struct K5Pre {      // M, G, X of one 32 x 32 slab: 8 steps of (4 rows x 32 colu
 template <int AMODE, int NMODE, int EPI, int XG>
 __global__ void __launch_bounds__(gemm_threads(AMODE, EPI), 1)
 gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArgs g) {
-    constexpr int NE = epi_warps(EPI);
+    constexpr int NE = epi_warps(AMODE, EPI);
     constexpr bool A_BUF = a_is_buf(AMODE);
     constexpr bool A_MN = (AMODE == A_IMG_MN || AMODE == A_BUF_COL);
     constexpr bool G_BF16 = (XG & 1) != 0;
@@ -706,7 +709,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 unsigned char* stg = staging + (warp - 2) * STAGING_BYTES_PER_WARP;
                 const int64_t gi0 = (int64_t)c.mt * BM + quarter * 32;
                 const int groups = (c.bn + 63) / 64;
-                for (int cg = 0; cg < groups; ++cg) {
+                for (int cg = (warp - 2) / 4; cg < groups; cg += NE / 4) {
                     const int valid = min(64, c.bn - cg * 64);          // multiple of 16
                     const int gj0 = c.n0 + cg * 64;
                     float f[64];
@@ -762,26 +765,41 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                         __syncwarp();
                     }
                     if (to_img) {
+                        // the two bf16 planes together (4 KB each in the staging buffer), then the fp16 plane
                         const int panel = gj0 / 64;
-                        for (int plane = 0; plane < d.img.planes; ++plane) {
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch) {
+                            const float fv[8] = {f[8 * ch], f[8 * ch + 1], f[8 * ch + 2], f[8 * ch + 3],
+                                                 f[8 * ch + 4], f[8 * ch + 5], f[8 * ch + 6], f[8 * ch + 7]};
+                            uint4 t0, t1;
+                            split8(fv, t0, t1);
+                            const int o = lane * 128 + img_chunk_offset(lane, ch);
+                            *reinterpret_cast<uint4*>(stg + o) = t0;
+                            *reinterpret_cast<uint4*>(stg + 4096 + o) = t1;
+                        }
+                        __syncwarp();
+                        unsigned char* dst0 = scr + img_row_offset(d.img, 0, panel, gi0);
+                        unsigned char* dst1 = scr + img_row_offset(d.img, 1, panel, gi0);
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            *reinterpret_cast<uint4*>(dst0 + it * 512 + lane * 16) =
+                                *reinterpret_cast<const uint4*>(stg + it * 512 + lane * 16);
+                            *reinterpret_cast<uint4*>(dst1 + it * 512 + lane * 16) =
+                                *reinterpret_cast<const uint4*>(stg + 4096 + it * 512 + lane * 16);
+                        }
+                        __syncwarp();
+                        if (d.img.planes == 3) {
 #pragma unroll
                             for (int ch = 0; ch < 8; ++ch) {
                                 const float fv[8] = {f[8 * ch], f[8 * ch + 1], f[8 * ch + 2], f[8 * ch + 3],
                                                      f[8 * ch + 4], f[8 * ch + 5], f[8 * ch + 6], f[8 * ch + 7]};
-                                uint4 t0, t1, out;
-                                if (plane == 2) {
-                                    out = half8(fv, 1.f);
-                                } else {
-                                    split8(fv, t0, t1);
-                                    out = plane == 0 ? t0 : t1;
-                                }
-                                *reinterpret_cast<uint4*>(stg + lane * 128 + img_chunk_offset(lane, ch)) = out;
+                                *reinterpret_cast<uint4*>(stg + lane * 128 + img_chunk_offset(lane, ch)) = half8(fv, 1.f);
                             }
                             __syncwarp();
-                            unsigned char* dst = scr + img_row_offset(d.img, plane, panel, gi0);
+                            unsigned char* dst2 = scr + img_row_offset(d.img, 2, panel, gi0);
 #pragma unroll
                             for (int it = 0; it < 8; ++it)
-                                *reinterpret_cast<uint4*>(dst + it * 512 + lane * 16) =
+                                *reinterpret_cast<uint4*>(dst2 + it * 512 + lane * 16) =
                                     *reinterpret_cast<const uint4*>(stg + it * 512 + lane * 16);
                             __syncwarp();
                         }
@@ -1376,7 +1394,7 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     while (cols < g.acc_bufs * accw) cols *= 2;
     g.tmem_cols = cols;
     const size_t fixed = (size_t)g.a_slots * g.a_slot_bytes +
-                         (tc::a_is_buf(AMODE) ? 0 : (size_t)tc::epi_warps(EPI) * g.epi_bufs * tc::STAGING_BYTES_PER_WARP) +
+                         (tc::a_is_buf(AMODE) ? 0 : (size_t)tc::epi_warps(AMODE, EPI) * g.epi_bufs * tc::STAGING_BYTES_PER_WARP) +
                          256 + 1024;
     g.n_slots = (int)std::min<size_t>(tc::MAX_N_SLOTS, (tc::SMEM_LIMIT - fixed) / (size_t)g.n_piece_bytes);
     // more than half of an SM's shared memory: one CTA per SM, whatever its tensor-memory share
