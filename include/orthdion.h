@@ -95,8 +95,11 @@ int orthdion_set_engine(orthdion_t h, int32_t engine);
  * split, about 2^-16 relative accuracy; 1 = one pass).  which: 0 = B*Q and B^T*P, 1 = Gram/apply
  * of the QR, 2 = P*R^T of the error feedback, 3 = P*Q^T of the weight update.  When both 2 and 3
  * ask for one pass, the fused pass runs in fp16 (11-bit operands, R scaled by a power of two);
- * otherwise a single pass means plain bf16.  Defaults: 3, 3, and 1, 1 for bf16 weights (3, 3 for
- * fp32 weights).  passes <= 0 restores the default. */
+ * otherwise a single pass means plain bf16.  Defaults: 3 and 3; for the fused pass 1, 1 with bf16
+ * weights while |b| <= 0.1 |a| (the momentum form), 3, 1 with bf16 weights otherwise (in the
+ * residual form a = b the fp16 error of P*R^T, about 4e-4, would show in M), 3, 3 with fp32
+ * weights.  The defaults follow later calls of set_dtypes and set_ef until a count is set here;
+ * passes <= 0 hands it back to the default rule. */
 int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes);
 
 /* Workspace sizes in bytes (host computation, no CUDA call). */

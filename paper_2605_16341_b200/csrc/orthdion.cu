@@ -27,6 +27,7 @@ struct orthdion_plan {
     float mu, eta, wd, scale, ef_a, ef_b;
     int32_t mode, x_dtype, g_dtype, engine;
     int32_t passes[4];
+    int32_t passes_set[4]; // 1: chosen by the caller, 0: follows the default rule
     int32_t diag;          // bit 0: factor diagnostics, bit 1: buffer norms (extra sweep over M, G)
 };
 
@@ -389,6 +390,18 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, cudaStrea
         if (c.p->diag) diag_stage(c, db, st);
 }
 
+// Default pass counts of the fused feedback/update pass.  One fp16 pass carries P R^T with about
+// 4e-4 relative error; in M' = a B - b P R^T that is harmless while b is small against a (the
+// momentum form, b = 1 - mu), but not in the residual form a = b, where M' is what is left after
+// the projection has been subtracted: then P R^T comes from split terms (three passes).
+void default_passes(orthdion_plan* p) {
+    const bool x32 = p->x_dtype == ORTHDION_DTYPE_F32;
+    if (!p->passes_set[0]) p->passes[0] = 3;
+    if (!p->passes_set[1]) p->passes[1] = 3;
+    if (!p->passes_set[2]) p->passes[2] = (x32 || std::fabs(p->ef_b) > 0.1f * std::fabs(p->ef_a)) ? 3 : 1;
+    if (!p->passes_set[3]) p->passes[3] = x32 ? 3 : 1;
+}
+
 int check_ptr(const void* p) {
     if (!p) return ORTHDION_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(p) % 16) return ORTHDION_ERR_ALIGNMENT;
@@ -415,7 +428,8 @@ int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r, float mu, 
     p->mode = mode;
     p->x_dtype = ORTHDION_DTYPE_BF16; p->g_dtype = ORTHDION_DTYPE_BF16;
     p->engine = tensor_engine_supports(m, n, r) ? ORTHDION_ENGINE_TENSOR : ORTHDION_ENGINE_SIMT;
-    p->passes[0] = 3; p->passes[1] = 3; p->passes[2] = 1; p->passes[3] = 1;
+    for (int k = 0; k < 4; ++k) p->passes_set[k] = 0;
+    default_passes(p);
     p->diag = 0;
     *out = p;
     return ORTHDION_OK;
@@ -434,10 +448,9 @@ int orthdion_set_dtypes(orthdion_t h, int32_t x_dtype, int32_t g_dtype) {
         (g_dtype != ORTHDION_DTYPE_F32 && g_dtype != ORTHDION_DTYPE_BF16))
         return ORTHDION_ERR_INVALID_ARG;
     h->x_dtype = x_dtype; h->g_dtype = g_dtype;
-    // bf16 weights: the fused feedback/update pass runs as one fp16 pass (11-bit operands: the
-    // feedback term b*P*R^T stays below 1e-5 of the buffer, the update is rounded to bf16 anyway).
-    // An fp32 weight matrix shows the update at full precision: both products from split terms.
-    h->passes[2] = h->passes[3] = (x_dtype == ORTHDION_DTYPE_F32) ? 3 : 1;
+    // bf16 weights: the update is rounded to bf16 anyway, one pass carries P Q^T.  An fp32 weight
+    // matrix shows the update at full precision: both products from split terms.
+    default_passes(h);
     return ORTHDION_OK;
 }
 
@@ -456,6 +469,7 @@ int orthdion_set_scale(orthdion_t h, float scale) {
 int orthdion_set_ef(orthdion_t h, float a, float b) {
     if (!valid(h) || !(a == a) || !(b == b)) return ORTHDION_ERR_INVALID_ARG;
     h->ef_a = a; h->ef_b = b;
+    default_passes(h);
     return ORTHDION_OK;
 }
 
@@ -471,11 +485,13 @@ int orthdion_set_engine(orthdion_t h, int32_t engine) {
 int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes) {
     if (!valid(h) || which < 0 || which > 3) return ORTHDION_ERR_INVALID_ARG;
     if (passes <= 0) {
-        passes = (which >= 2) ? (h->x_dtype == ORTHDION_DTYPE_F32 ? 3 : 1) : 3;
-    } else if (passes != 1 && passes != 3) {
-        return ORTHDION_ERR_INVALID_ARG;
+        h->passes_set[which] = 0;
+        default_passes(h);
+        return ORTHDION_OK;
     }
+    if (passes != 1 && passes != 3) return ORTHDION_ERR_INVALID_ARG;
     h->passes[which] = passes;
+    h->passes_set[which] = 1;
     return ORTHDION_OK;
 }
 

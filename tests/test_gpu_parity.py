@@ -151,6 +151,17 @@ def test_paper_error_feedback_form_and_decay(engine):
     one_step_compare(spec, X, M, G, Q, mode=od.MODE_ORTH, engine=engine, wd=0.1, scale=0.5, eta=0.02)
 
 
+# ------------------------------------------------------------------ the paper's own shape classes
+@pytest.mark.parametrize("shape", [(768, 768, 192), (768, 2048, 192), (2048, 768, 192)])
+@pytest.mark.parametrize("mode", MODES)
+def test_shape_classes_of_the_320m_model(shape, mode):
+    # hidden width 768, MLP width 2048, rank fraction 0.25 of the smaller side, the paper's
+    # error-feedback form (beta, beta) and its learning rate and weight decay
+    m, n, r = shape
+    spec, X, M, G, Q = make_problem(m, n, r, BF16, BF16, seed=m + 3 * n)
+    one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_TENSOR, ef=(0.95, 0.95), eta=0.012, wd=0.1)
+
+
 # ------------------------------------------------------------------ degenerate inputs
 @pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
 def test_zero_buffer_is_flagged_and_state_untouched(engine):
