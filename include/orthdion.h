@@ -71,8 +71,9 @@ typedef struct orthdion_plan* orthdion_t;
 #define ORTHDION_ERR_ALIGNMENT     -6   /* a matrix pointer is not 16-byte aligned              */
 
 /* per-matrix device status flags (bit mask) */
-#define ORTHDION_STATUS_SHIFTED_LEFT    1   /* left QR took the shifted three-pass path         */
-#define ORTHDION_STATUS_SHIFTED_RIGHT   2   /* right QR took the shifted three-pass path        */
+#define ORTHDION_STATUS_SHIFTED_LEFT    1   /* left QR took three passes (shifted first pass,   */
+#define ORTHDION_STATUS_SHIFTED_RIGHT   2   /* or a second pass that met a poorly conditioned   */
+                                            /* Q1); same for the right QR                       */
 #define ORTHDION_STATUS_RANK_DEFICIENT  4   /* factorisation failed: X, M, Q left unchanged     */
 #define ORTHDION_STATUS_NONFINITE       8   /* a Gram matrix held Inf/NaN: treated as failure   */
 #define ORTHDION_STATUS_ZERO_COLUMN    16   /* COLNORM met a zero column of R (kept zero)       */

@@ -30,6 +30,7 @@ constexpr int CT_NB = 32;
 constexpr int CT_KC = 32;             // depth of one staged chunk
 constexpr int CT_LDK = 40;            // staged rows: 32 bf16 + 8 of padding (conflict-free fragment loads)
 constexpr int CT_MAX_TASKS = 160;
+constexpr float CT_THIRD_PASS_LIMIT = 0.02f; // bound on |Gram - I|_2 of the second pass above which a third follows
 constexpr float CT_SERIES_LIMIT = 1.4e-3f;   // bound on |Gram - I|_2 below which L^{-1} = I - Phi(E) is used
 
 // C(i,j) = beta*C(i,j) + alpha * sum_{k in [kbeg,kend)} A(i,k) B(k,j), i < Mt <= 64, j < Nt <= 64.
@@ -316,6 +317,9 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         mx = 0.f;
         for (int i = 0; i < CT_THREADS / 32; ++i) mx = fmaxf(mx, red[i]);
         series = mx <= CT_SERIES_LIMIT;          // false for NaN
+        // Second pass with Q1 far from orthonormal (cond(Y)^2 u was not small): its result will
+        // not be orthonormal to working accuracy either, so ask for the third pass.
+        if (a.pass == 2 && !(mx <= CT_THIRD_PASS_LIMIT) && tid == 0) atomicOr(w.status, shift_bit);
         __syncthreads();
     }
     if (series) {

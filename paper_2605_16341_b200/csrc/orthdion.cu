@@ -37,7 +37,11 @@ constexpr uint32_t kMagic = 0x0D10A5E7u;
 constexpr int32_t kMaxRank = 1024;
 constexpr size_t kScratchBudget = (size_t)24 << 30;   // per launch batch
 constexpr float kShiftRel = 1e-5f;
+// max/min diag(L) of the first Cholesky above which the QR takes the shifted three-pass path.
+// CholeskyQR2 needs cond(Y)^2 * u well below 1, u the accuracy of the Gram/apply products:
+// fp32 for the SIMT engine, about 2^-16 for the split-bf16 products of the tensor engine.
 constexpr float kCondLimit = 1024.f;
+constexpr float kCondLimitTensor = 96.f;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool valid(orthdion_t h) { return h && h->magic == kMagic; }
@@ -194,7 +198,8 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
         const int r = lead.p->r;
         CholArgs ca{};
         ca.gram = sel(W_SCRATCH, lead.sc.gram); ca.work = sel(W_SCRATCH, lead.sc.linv);
-        ca.r = r; ca.which = which; ca.pass = pass; ca.shift_rel = kShiftRel; ca.cond_limit = kCondLimit;
+        ca.r = r; ca.which = which; ca.pass = pass; ca.shift_rel = kShiftRel;
+        ca.cond_limit = lead.tensor() ? kCondLimitTensor : kCondLimit;
         ca.colsq = sel(W_SCRATCH, 0); ca.use_colsq = 0; ca.img = no_img(); ca.cnorm_off = -1;
         if (lead.tensor()) {
             ca.colsq = sel(W_SCRATCH, lead.sc.ts.colsq); ca.use_colsq = 1; ca.img = lead.sc.ts.linv;

@@ -103,7 +103,7 @@ def test_cfg0_chained_both_modes(engine):
 # ------------------------------------------------------------------ one step, several shapes
 SHAPES_ANY = [(200, 328, 24), (129, 520, 8), (64, 64, 64), (520, 136, 40), (96, 1000, 1), (300, 77, 5)]
 SHAPES_TENSOR = [(256, 512, 16), (384, 640, 64), (200, 328, 48), (1000, 264, 128), (136, 2056, 32),
-                 (640, 384, 272)]
+                 (640, 384, 272), (64, 64, 64), (96, 1000, 16), (48, 136, 16), (16, 16, 16)]
 
 
 @pytest.mark.parametrize("shape", SHAPES_ANY)
@@ -117,7 +117,7 @@ def test_one_step_simt_shapes(shape, mode, dt):
 
 @pytest.mark.parametrize("shape", SHAPES_TENSOR)
 @pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("dt", [(F32, F32), (BF16, BF16), (F32, BF16)])
+@pytest.mark.parametrize("dt", [(F32, F32), (BF16, BF16), (F32, BF16), (BF16, F32)])
 def test_one_step_tensor_shapes(shape, mode, dt):
     m, n, r = shape
     spec, X, M, G, Q = make_problem(m, n, r, dt[0], dt[1], seed=m * 7 + n)
