@@ -575,6 +575,12 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                             // (rows beyond the matrix are zero in the images; those columns of D are never stored)
                             const uint32_t ncols = (uint32_t)((min(128, c.bn - ch * 128) + 15) / 16 * 16);
                             const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u, fmt);
+                            // Fused pass with single-term operands: the R piece and the Q piece lie back
+                            // to back in the slot (256 rows of one K-major tile) and their accumulators in
+                            // adjacent columns, so one N = 256 instruction serves both products and reads
+                            // the P slice from shared memory once.
+                            const bool both = EPI == EPI_K5 && g.passes == 1 && g.passes2 == 1 && ncols == 128 && g.BN == 128;
+                            const uint32_t idesc2 = instr_desc(256u, A_MN ? 1u : 0u, 0u, fmt);
                             // (Descriptors are rebuilt per instruction here on purpose: with the additive
                             // form of the other branch the fused pass measured 38 ms instead of 26 ms per
                             // step; its N = 128 instructions run best when they are not issued back to back.)
@@ -587,6 +593,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                 const uint64_t b1 = smem_desc(sn + A_TERM_BYTES + j * 32, 16, 1024);
                                 const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
                                 const uint32_t d1 = dacc + ch * 128;
+                                if (both) { umma_bf16(d1, a0, b0, idesc2, accum); continue; }
                                 umma_bf16(d1, a0, b0, idesc, accum);
                                 if (g.passes == 3) {
                                     umma_bf16(d1, a0, b1, idesc, 1u);
