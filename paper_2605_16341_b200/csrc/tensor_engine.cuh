@@ -78,7 +78,8 @@ struct GemmArgs {
     int32_t tmem_cols;                       // allocation (power of two >= 32)
     int32_t fp16;                            // single-pass fp16 products from plane 2 of the images
     int32_t a_slots, a_slot_bytes;           // A ring
-    int32_t epi_bufs, pad1;                  // fused pass: 8 KB epilogue buffers per warp (1 or 2)
+    int32_t epi_bufs;                        // fused pass: 8 KB epilogue buffers per warp (1 or 2)
+    int32_t pair;                            // launched as CTA pairs (clusters of two, M = 256 instructions)
     int64_t rscale_off;                      // fp16 fused pass: scratch offset of 1 / (scale of R's plane)
     int64_t ld;                              // leading dimension of M, G, X
     ImgRef a, n1, n2;
@@ -138,6 +139,70 @@ __device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* ma
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(panel), "r"(plane), "r"(matrix), "r"(bar)
         : "memory");
 }
+// ---- CTA pairs (clusters of two CTAs on neighbouring SMs, tcgen05 cta_group::2) ----------------
+// One MMA instruction of the pair's leader (cluster rank 0) multiplies M = 256 rows: each CTA
+// supplies its own 128 rows of A and HALF of the N-side operand, and receives its 128 rows of the
+// result in its own tensor memory.  Per CTA that halves the N-side bytes that are fetched from L2
+// and read from shared memory by the tensor core.  Barriers that gather both CTAs (operand
+// "full", accumulator "empty") live in the leader and are reached by remote arrives; barriers
+// that release (operand "empty", accumulator "full") live in each CTA and are reached by the
+// leader's multicast commit.  All of them keep the default (CTA-scope) semantics of the single-CTA
+// barriers: with release/acquire at cluster scope on every arrive and wait the same kernels ran up
+// to twice as long (the producer thread then pays a cluster-wide fence per load).
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the location `addr` (a shared::cta address) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_remote(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;"
+                 ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Tiled TMA load of a CTA of a pair: the data lands in this CTA's shared memory, the bytes are
+// counted on the mbarrier at cluster address `bar` (the leader's).
+__device__ __forceinline__ void tma_load_box_pair(uint32_t dst, const CUtensorMap* map, int row, int panel, int plane,
+                                                  int matrix, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(panel), "r"(plane), "r"(matrix), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T with M = 256; issued by one thread of the leader.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the mbarrier at offset `bar` of BOTH CTAs arrives once every MMA issued so far has completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
 // Asynchronous 16-byte copy global -> shared (no register staging), grouped per thread.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -195,9 +260,22 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 // Instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = n; a_mn / b_mn = 1 for an
 // MN-major A / B operand (0: K-major).
 // fmt: operand format, 1 = bf16, 0 = fp16 (both operands alike).
-__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t a_mn, uint32_t b_mn, uint32_t fmt = 1u) {
+// m: rows of the instruction, 128, or 256 for an instruction of a CTA pair.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t a_mn, uint32_t b_mn, uint32_t fmt = 1u,
+                                               uint32_t m = (uint32_t)BM) {
     return (1u << 4) | (fmt << 7) | (fmt << 10) | (a_mn << 15) | (b_mn << 16) | ((n >> 3) << 17) |
-           ((uint32_t)(BM >> 4) << 24);
+           ((m >> 4) << 24);
+}
+template <bool PAIR>
+__device__ __forceinline__ void umma_any(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    if (PAIR) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, accumulate);
+    else umma_bf16(d_tmem, adesc, bdesc, idesc, accumulate);
+}
+template <bool PAIR>
+__device__ __forceinline__ void commit_any(uint32_t bar) {
+    if (PAIR) umma_commit_pair(bar);
+    else umma_commit(bar);
 }
 
 __device__ __forceinline__ void load8(const void* base, int64_t idx, int is_bf16, float (&v)[8]) {
@@ -317,14 +395,19 @@ struct TileCoord { int b, mt, nt, n0, bn, kb_end; bool active; };
 // the kernel runs), so that only the first tile of a matrix pays for the global load.
 struct StatusCache { int b = -1; int st = 0; };
 
+// Pair launches (g.pair): a scheduled row tile is 256 rows, CTA `rank` of the pair owns its
+// rows 128 * rank .. ; c.mt stays the 128-row tile index (it may lie one past the last tile when
+// the number of tiles is odd: that CTA multiplies zeros and stores nothing).
 template <int EPI>
-__device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmArgs& g, int t, StatusCache& sc) {
+__device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmArgs& g, int t, StatusCache& sc,
+                                                 int rank) {
     TileCoord c;
     const int per = g.m_tiles * g.n_tiles;
     c.b = t / per;
     const int rem = t - c.b * per;
-    c.mt = rem / g.n_tiles;
-    c.nt = rem - c.mt * g.n_tiles;
+    const int mts = rem / g.n_tiles;
+    c.nt = rem - mts * g.n_tiles;
+    c.mt = g.pair ? 2 * mts + rank : mts;
     c.n0 = c.nt * g.BN;
     c.bn = min(g.BN, g.Ncols - c.n0);
     c.kb_end = g.k_blocks;
@@ -333,7 +416,7 @@ __device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmA
     const int st = sc.st;
     c.active = !(st & ST_FAILED);
     if (EPI != EPI_K5 && g.out.only_if_shifted && !(st & g.out.shift_bit)) c.active = false;
-    if (g.lower_only && c.n0 > c.mt * BM + BM - 1) c.active = false;
+    if (g.lower_only && c.n0 > (g.pair ? 2 * mts + 1 : c.mt) * BM + BM - 1) c.active = false;
     return c;
 }
 
@@ -371,10 +454,14 @@ struct K5Pre {      // M, G, X of one 32 x 32 slab: 8 steps of (4 rows x 32 colu
     uint32_t x[8][(XG & 2) ? 2 : 4];
 };
 
-template <int AMODE, int NMODE, int EPI, int XG>
+template <int AMODE, int NMODE, int EPI, int XG, bool PAIR>
 __global__ void __launch_bounds__(gemm_threads(AMODE, EPI), 1)
 gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArgs g) {
     constexpr int NE = epi_warps(AMODE, EPI);
+    // PAIR: launched in clusters of two; rank 0 (the leader) issues every MMA for both CTAs
+    const int crank = PAIR ? (int)cluster_ctarank() : 0;
+    const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int tstride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     constexpr bool A_BUF = a_is_buf(AMODE);
     constexpr bool A_MN = (AMODE == A_IMG_MN || AMODE == A_BUF_COL);
     constexpr bool G_BF16 = (XG & 1) != 0;
@@ -397,27 +484,38 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     StatusCache scache;
 
+    // Pairs: the "full" barriers of the operand rings and the "empty" barriers of the accumulators
+    // that are used are the leader's; they count the arrivals of both CTAs.
+    constexpr uint32_t NCTA = PAIR ? 2u : 1u;
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_A_SLOTS; ++s) {
-            mbar_init(a_full0 + 8 * s, A_BUF ? NUM_XF_WARPS : 1);
+            mbar_init(a_full0 + 8 * s, NCTA * (A_BUF ? NUM_XF_WARPS : 1));
             mbar_init(a_empty0 + 8 * s, 1);
         }
         for (int s = 0; s < MAX_N_SLOTS; ++s) {
-            mbar_init(n_full0 + 8 * s, 1);
+            mbar_init(n_full0 + 8 * s, NCTA);
             mbar_init(n_empty0 + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull0 + 8 * a, 1);
-            mbar_init(tempty0 + 8 * a, NE);
+            mbar_init(tempty0 + 8 * a, NCTA * NE);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)g.tmem_cols);
+    if (warp == 1) {
+        if (PAIR) tmem_alloc_pair(smem_u32(tmem_slot), (uint32_t)g.tmem_cols);
+        else tmem_alloc(smem_u32(tmem_slot), (uint32_t)g.tmem_cols);
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();       // the peer's barriers are initialised before anything reaches them
     tc_fence_after();
+    // cluster addresses of the leader's gathering barriers (slot s: + 8 s)
+    const uint32_t a_full_ld = PAIR ? map_to_rank(a_full0, 0) : a_full0;
+    const uint32_t n_full_ld = PAIR ? map_to_rank(n_full0, 0) : n_full0;
+    const uint32_t tempty_ld = PAIR ? map_to_rank(tempty0, 0) : tempty0;
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t acc_stride = (uint32_t)(g.tmem_cols / g.acc_bufs);
 
@@ -427,7 +525,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     const uint32_t fmt = g.fp16 ? 0u : 1u;
     // N_IMG_MN piece geometry: [term][64-column group][ks rows of 128 bytes]
     const uint32_t group_stride = (uint32_t)g.ks * 128u;
-    const uint32_t mn_term_stride = (uint32_t)((g.BN + 63) / 64) * group_stride;
+    const uint32_t mn_term_stride = PAIR ? 2u * group_stride : (uint32_t)((g.BN + 63) / 64) * group_stride;
 
     if (warp == 0) {
         // ---------------- producer ----------------
@@ -438,23 +536,23 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         if (lane == 0) {
             int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
             // cursor over (tile, depth block) for the A ring
-            int at = blockIdx.x, akb = 0; TileCoord ac{}; bool a_done = A_BUF;
+            int at = tile0, akb = 0; TileCoord ac{}; bool a_done = A_BUF;
             // cursor over (tile, depth block, piece) for the N ring
-            int nt_ = blockIdx.x, nkb = 0, npc = 0; TileCoord nc{}; bool n_done = false;
+            int nt_ = tile0, nkb = 0, npc = 0; TileCoord nc{}; bool n_done = false;
             auto a_seek = [&]() {           // make (at, akb) valid or finish
                 while (!a_done) {
                     if (at >= g.total_tiles) { a_done = true; break; }
-                    if (akb == 0) ac = decode_tile<EPI>(batch, g, at, scache);
+                    if (akb == 0) ac = decode_tile<EPI>(batch, g, at, scache, crank);
                     if (ac.active && akb < ac.kb_end) break;
-                    at += gridDim.x; akb = 0;
+                    at += tstride; akb = 0;
                 }
             };
             auto n_pieces = [&](int kb) { return NMODE == N_IMG_MN ? mn_pieces(g, kb) : (nc.bn + 127) / 128; };
             auto n_seek = [&]() {           // make (nt_, nkb, npc) valid or finish
                 while (!n_done) {
                     if (nt_ >= g.total_tiles) { n_done = true; break; }
-                    if (nkb == 0 && npc == 0) nc = decode_tile<EPI>(batch, g, nt_, scache);
-                    if (!nc.active || nkb >= nc.kb_end) { nt_ += gridDim.x; nkb = 0; npc = 0; continue; }
+                    if (nkb == 0 && npc == 0) nc = decode_tile<EPI>(batch, g, nt_, scache, crank);
+                    if (!nc.active || nkb >= nc.kb_end) { nt_ += tstride; nkb = 0; npc = 0; continue; }
                     if (npc >= n_pieces(nkb)) { ++nkb; npc = 0; continue; }
                     if (NMODE == N_IMG_K && !k_piece_active(g, nc, nkb, npc)) { ++npc; continue; }
                     break;
@@ -466,27 +564,43 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             while (!a_done || !n_done) {
                 bool progress = false;
                 if (!a_done && mbar_try_wait(a_empty0 + 8 * as, aph ^ 1)) {
-                    const uint32_t fb = a_full0 + 8 * as;
                     const uint32_t dst = smem_u32(a_ring + as * g.a_slot_bytes);
-                    mbar_arrive_expect_tx(fb, (uint32_t)a_terms * A_TERM_BYTES);
-                    if (AMODE == A_IMG_K) tma_load_box(dst, &g.map_a, ac.mt * BM, akb, plane, ac.b, fb);
-                    else tma_load_box(dst, &g.map_a, akb * BK, ac.mt * 2, plane, ac.b, fb);
+                    if (PAIR) {
+                        const uint32_t fb = a_full_ld + 8 * as;
+                        mbar_arrive_expect_tx_remote(fb, (uint32_t)a_terms * A_TERM_BYTES);
+                        if (AMODE == A_IMG_K) tma_load_box_pair(dst, &g.map_a, ac.mt * BM, akb, plane, ac.b, fb);
+                        else tma_load_box_pair(dst, &g.map_a, akb * BK, ac.mt * 2, plane, ac.b, fb);
+                    } else {
+                        const uint32_t fb = a_full0 + 8 * as;
+                        mbar_arrive_expect_tx(fb, (uint32_t)a_terms * A_TERM_BYTES);
+                        if (AMODE == A_IMG_K) tma_load_box(dst, &g.map_a, ac.mt * BM, akb, plane, ac.b, fb);
+                        else tma_load_box(dst, &g.map_a, akb * BK, ac.mt * 2, plane, ac.b, fb);
+                    }
                     if (++as == g.a_slots) { as = 0; aph ^= 1; }
                     ++akb;
-                    if (akb >= ac.kb_end) { at += gridDim.x; akb = 0; }
+                    if (akb >= ac.kb_end) { at += tstride; akb = 0; }
                     a_seek();
                     progress = true;
                 }
                 if (!n_done && mbar_try_wait(n_empty0 + 8 * ns, nph ^ 1)) {
-                    const uint32_t fb = n_full0 + 8 * ns;
+                    const uint32_t fb = PAIR ? n_full_ld + 8 * ns : n_full0 + 8 * ns;
                     const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
-                    mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
-                    if (NMODE == N_IMG_MN) {
-                        tma_load_box(dst, &g.map_n1, nkb * BK + npc * g.ks, nc.n0 / 64, plane, nc.b, fb);
+                    if (PAIR) {
+                        // this CTA's half of the N-side: per 256-column block its two 64-column groups
+                        mbar_arrive_expect_tx_remote(fb, (uint32_t)g.n_piece_bytes);
+                        const uint32_t blk_bytes = (uint32_t)n1_terms * 2u * group_stride;
+                        for (int blk = 0; blk * 256 < nc.bn; ++blk)
+                            tma_load_box_pair(dst + blk * blk_bytes, &g.map_n1, nkb * BK + npc * g.ks,
+                                              nc.n0 / 64 + blk * 4 + crank * 2, plane, nc.b, fb);
                     } else {
-                        tma_load_box(dst, &g.map_n1, nc.n0 + npc * 128, nkb, plane, nc.b, fb);
-                        if (EPI == EPI_K5)
-                            tma_load_box(dst + n1_terms * A_TERM_BYTES, &g.map_n2, nc.n0 + npc * 128, nkb, plane, nc.b, fb);
+                        mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
+                        if (NMODE == N_IMG_MN) {
+                            tma_load_box(dst, &g.map_n1, nkb * BK + npc * g.ks, nc.n0 / 64, plane, nc.b, fb);
+                        } else {
+                            tma_load_box(dst, &g.map_n1, nc.n0 + npc * 128, nkb, plane, nc.b, fb);
+                            if (EPI == EPI_K5)
+                                tma_load_box(dst + n1_terms * A_TERM_BYTES, &g.map_n2, nc.n0 + npc * 128, nkb, plane, nc.b, fb);
+                        }
                     }
                     if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
                     ++npc;
@@ -521,8 +635,11 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         const uint32_t a_ring16 = smem_u32(a_ring) >> 4, n_ring16 = smem_u32(n_ring) >> 4;
         const uint32_t a_slot16 = (uint32_t)g.a_slot_bytes >> 4, n_slot16 = (uint32_t)g.n_piece_bytes >> 4;
         const bool three = g.passes == 3;
-        for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-            const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+        constexpr uint32_t MROWS = PAIR ? 256u : 128u;
+        // pairs: a 256-column block of the N-side is this CTA's two 64-column groups, both terms
+        const uint32_t n_block16 = (PAIR ? (uint32_t)n1_terms * 2u * group_stride : 4u * group_stride) >> 4;
+        for (int t = tile0; t < g.total_tiles && ok && crank == 0; t += tstride) {
+            const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
             if (!c.active) continue;
             if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -547,16 +664,16 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                 const uint32_t accum = (kb > 0 || sub > 0 || j > 0) ? 1u : 0u;
                                 uint64_t b0 = n_pc + (uint32_t)j * n_slice16;
                                 for (int cc = 0; cc < c.bn; cc += 256) {
-                                    const uint32_t idesc = instr_desc((uint32_t)min(256, c.bn - cc), A_MN ? 1u : 0u, 1u, fmt);
-                                    umma_bf16(dacc + cc, a0, b0, idesc, accum);
+                                    const uint32_t idesc = instr_desc((uint32_t)min(256, c.bn - cc), A_MN ? 1u : 0u, 1u, fmt, MROWS);
+                                    umma_any<PAIR>(dacc + cc, a0, b0, idesc, accum);
                                     if (three) {
-                                        umma_bf16(dacc + cc, a0, b0 + n_term16, idesc, 1u);
-                                        umma_bf16(dacc + cc, a1, b0, idesc, 1u);
+                                        umma_any<PAIR>(dacc + cc, a0, b0 + n_term16, idesc, 1u);
+                                        umma_any<PAIR>(dacc + cc, a1, b0, idesc, 1u);
                                     }
-                                    b0 += 4 * (group_stride >> 4);          // next 256 columns: four 64-column groups
+                                    b0 += n_block16;                        // next 256 columns
                                 }
                             }
-                            umma_commit(n_empty0 + 8 * ns);
+                            commit_any<PAIR>(n_empty0 + 8 * ns);
                         }
                         __syncwarp();
                         if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
@@ -574,13 +691,13 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                             // N of the instruction must be a multiple of 16: round a ragged last chunk up
                             // (rows beyond the matrix are zero in the images; those columns of D are never stored)
                             const uint32_t ncols = (uint32_t)((min(128, c.bn - ch * 128) + 15) / 16 * 16);
-                            const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u, fmt);
+                            const uint32_t idesc = instr_desc(ncols, A_MN ? 1u : 0u, 0u, fmt, MROWS);
                             // Fused pass with single-term operands: the R piece and the Q piece lie back
                             // to back in the slot (256 rows of one K-major tile) and their accumulators in
                             // adjacent columns, so one N = 256 instruction serves both products and reads
                             // the P slice from shared memory once.
                             const bool both = EPI == EPI_K5 && g.passes == 1 && g.passes2 == 1 && ncols == 128 && g.BN == 128;
-                            const uint32_t idesc2 = instr_desc(256u, A_MN ? 1u : 0u, 0u, fmt);
+                            const uint32_t idesc2 = instr_desc(256u, A_MN ? 1u : 0u, 0u, fmt, MROWS);
                             // (Descriptors are rebuilt per instruction here on purpose: with the additive
                             // form of the other branch the fused pass measured 38 ms instead of 26 ms per
                             // step; its N = 128 instructions run best when they are not issued back to back.)
@@ -593,37 +710,37 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                 const uint64_t b1 = smem_desc(sn + A_TERM_BYTES + j * 32, 16, 1024);
                                 const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
                                 const uint32_t d1 = dacc + ch * 128;
-                                if (both) { umma_bf16(d1, a0, b0, idesc2, accum); continue; }
-                                umma_bf16(d1, a0, b0, idesc, accum);
+                                if (both) { umma_any<PAIR>(d1, a0, b0, idesc2, accum); continue; }
+                                umma_any<PAIR>(d1, a0, b0, idesc, accum);
                                 if (g.passes == 3) {
-                                    umma_bf16(d1, a0, b1, idesc, 1u);
-                                    umma_bf16(d1, a1, b0, idesc, 1u);
+                                    umma_any<PAIR>(d1, a0, b1, idesc, 1u);
+                                    umma_any<PAIR>(d1, a1, b0, idesc, 1u);
                                 }
                                 if (EPI == EPI_K5) {
                                     const uint32_t s2 = sn + n1_terms * A_TERM_BYTES;
                                     const uint64_t c0 = smem_desc(s2 + j * 32, 16, 1024);
                                     const uint64_t c1 = smem_desc(s2 + A_TERM_BYTES + j * 32, 16, 1024);
                                     const uint32_t d2 = dacc + g.BN;
-                                    umma_bf16(d2, a0, c0, idesc, accum);
+                                    umma_any<PAIR>(d2, a0, c0, idesc, accum);
                                     if (g.passes2 == 3) {
-                                        umma_bf16(d2, a0, c1, idesc, 1u);
-                                        umma_bf16(d2, a1, c0, idesc, 1u);
+                                        umma_any<PAIR>(d2, a0, c1, idesc, 1u);
+                                        umma_any<PAIR>(d2, a1, c0, idesc, 1u);
                                     }
                                 }
                             }
-                            umma_commit(n_empty0 + 8 * ns);
+                            commit_any<PAIR>(n_empty0 + 8 * ns);
                         }
                         __syncwarp();
                         if (++ns == g.n_slots) { ns = 0; nph ^= 1; }
                     }
                 }
                 if (!ok) break;
-                if (lane == 0) umma_commit(a_empty0 + 8 * as);
+                if (lane == 0) commit_any<PAIR>(a_empty0 + 8 * as);
                 __syncwarp();
                 if (++as == g.a_slots) { as = 0; aph ^= 1; }
             }
             if (!ok) break;
-            if (lane == 0) umma_commit(tfull0 + 8 * acc);
+            if (lane == 0) commit_any<PAIR>(tfull0 + 8 * acc);
             __syncwarp();
             if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
         }
@@ -633,8 +750,8 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         bool ok = true;
         const int quarter = warp % 4;                    // tensor-memory lanes 32*quarter .. +31
         if (EPI == EPI_STORE) {
-            for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-                const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+            for (int t = tile0; t < g.total_tiles && ok; t += tstride) {
+                const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
                 if (!c.active) continue;
                 if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -651,7 +768,9 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 // One wide tile per long main loop: the epilogue is a small share of the time, so
                 // it stores row per lane, 16 columns at a time, straight from the registers.
                 const int64_t gi = (int64_t)c.mt * BM + quarter * 32 + lane;
-                const int bn64 = to_img ? (c.bn + 63) / 64 * 64 : c.bn;
+                // (pairs: the CTA whose rows lie beyond the matrix stores nothing)
+                const bool has_rows = !PAIR || (int64_t)c.mt * BM < g.Mrows;
+                const int bn64 = !has_rows ? 0 : (to_img ? (c.bn + 63) / 64 * 64 : c.bn);
                 for (int cc = 0; cc < bn64; cc += 16) {
                     uint32_t v[16];
                     if (cc < c.bn) {
@@ -715,7 +834,8 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 // 128 bytes, byte for byte what the image holds, so it leaves as one 4 KB run.
                 unsigned char* stg = staging + (warp - 2) * STAGING_BYTES_PER_WARP;
                 const int64_t gi0 = (int64_t)c.mt * BM + quarter * 32;
-                const int groups = (c.bn + 63) / 64;
+                const bool has_rows = !PAIR || (int64_t)c.mt * BM < g.Mrows;
+                const int groups = has_rows ? (c.bn + 63) / 64 : 0;
                 for (int cg = (warp - 2) / 4; cg < groups; cg += NE / 4) {
                     const int valid = min(64, c.bn - cg * 64);          // multiple of 16
                     const int gj0 = c.n0 + cg * 64;
@@ -815,7 +935,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                if (lane == 0) { if (PAIR) mbar_arrive_remote(tempty_ld + 8 * acc); else mbar_arrive(tempty0 + 8 * acc); }
                 if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
             }
         } else {
@@ -826,8 +946,8 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             // tile's M, G, X in L2, so the loads of a slab return with L2 latency.
             const int half = (warp - 2) / 4;
             auto next_tile = [&](int t) {
-                for (t += gridDim.x; t < g.total_tiles; t += gridDim.x)
-                    if (decode_tile<EPI>(batch, g, t, scache).active) return t;
+                for (t += tstride; t < g.total_tiles; t += tstride)
+                    if (decode_tile<EPI>(batch, g, t, scache, crank).active) return t;
                 return g.total_tiles;
             };
             // the slabs of this warp in order: (tile, 0), (tile, 1), (next tile, 0), ...
@@ -848,7 +968,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 auto m_off = [](int r, int ch) { return r * 128 + ((ch ^ (r & 7)) << 4); };
                 auto h_off = [](int r, int ch) { return r * 64 + ((ch ^ ((r >> 1) & 3)) << 4); };
                 auto issue = [&](int t, int slab, unsigned char* buf) {
-                    const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+                    const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
                     const MatWork& w = batch.w[c.b];
                     const int64_t gj0 = (int64_t)c.n0 + half * 64 + slab * 32;
                     const int64_t gi0 = (int64_t)c.mt * BM + quarter * 32;
@@ -872,7 +992,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                     cp_async_commit();
                 };
                 auto process = [&](int t, int slab, unsigned char* buf) -> bool {
-                    const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+                    const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
                     const MatWork& w = batch.w[c.b];
                     const float efb = g.fp16 ? g.ef_b * *reinterpret_cast<const float*>(w.scratch + g.rscale_off) : g.ef_b;
                     if (slab == 0) {
@@ -925,7 +1045,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                         // the accumulators of this tile are in registers / shared memory now
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                        if (lane == 0) { if (PAIR) mbar_arrive_remote(tempty_ld + 8 * acc); else mbar_arrive(tempty0 + 8 * acc); }
                         if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
                     }
                     __syncwarp();
@@ -949,7 +1069,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                     __syncwarp();
                     return true;
                 };
-                int t = next_tile(blockIdx.x - (int)gridDim.x), slab = 0, ib = 0;
+                int t = next_tile(tile0 - tstride), slab = 0, ib = 0;
                 if (t < g.total_tiles) issue(t, slab, bufs);
                 while (t < g.total_tiles) {
                     int t2 = t, slab2 = slab;
@@ -974,7 +1094,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             const int rl = lane / 8, cq = lane % 8;      // row within a step, 4-column group
 
             auto fetch = [&](K5Pre<XG>& p, int t, int slab) {
-                const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+                const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
                 const MatWork& w = batch.w[c.b];
                 const int64_t gj = (int64_t)c.n0 + half * 64 + slab * 32 + cq * 4;
 #pragma unroll
@@ -1003,7 +1123,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
 
             // one slab: accumulators -> staging -> row-wise update of M and X
             auto process = [&](const K5Pre<XG>& cur, int t, int slab) -> bool {
-                const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+                const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
                 const MatWork& w = batch.w[c.b];
                 const float efb = g.fp16 ? g.ef_b * *reinterpret_cast<const float*>(w.scratch + g.rscale_off) : g.ef_b;
                 if (slab == 0) {
@@ -1079,12 +1199,12 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 if (slab == 1) {
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+                    if (lane == 0) { if (PAIR) mbar_arrive_remote(tempty_ld + 8 * acc); else mbar_arrive(tempty0 + 8 * acc); }
                     if (++acc == g.acc_bufs) { acc = 0; acc_phase ^= 1; }
                 }
                 return true;
             };
-            int t = next_tile(blockIdx.x - (int)gridDim.x), slab = 0;
+            int t = next_tile(tile0 - tstride), slab = 0;
             K5Pre<XG> pa;
             while (t < g.total_tiles) {
                 fetch(pa, t, slab);
@@ -1101,8 +1221,8 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         int as = 0; uint32_t aph = 0;
         bool ok = true;
         struct Raw { float4 m[2][2]; uint32_t gq[2][G_BF16 ? 4 : 8]; };
-        for (int t = blockIdx.x; t < g.total_tiles && ok; t += gridDim.x) {
-            const TileCoord c = decode_tile<EPI>(batch, g, t, scache);
+        for (int t = tile0; t < g.total_tiles && ok; t += tstride) {
+            const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
             if (!c.active) continue;
             const MatWork& w = batch.w[c.b];
             const int64_t ld = g.ld;
@@ -1182,7 +1302,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(a_full0 + 8 * as);
+                if (lane == 0) { if (PAIR) mbar_arrive_remote(a_full_ld + 8 * as); else mbar_arrive(a_full0 + 8 * as); }
                 if (++as == g.a_slots) { as = 0; aph ^= 1; }
                 return true;
             };
@@ -1206,11 +1326,16 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     // ---------------- teardown ----------------
     tc_fence_before();
     __syncthreads();
+    // pairs: neither CTA leaves (or frees tensor memory) while the other may still reach its barriers
+    if (PAIR) cluster_sync_all();
     tc_fence_after();
     if (*abort_flag && threadIdx.x == 0) {
         for (int b = 0; b < batch.count; ++b) atomicOr(batch.w[b].status, ST_WAIT);
     }
-    if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)g.tmem_cols);
+    if (warp == 1) {
+        if (PAIR) tmem_dealloc_pair(tmem_base, (uint32_t)g.tmem_cols);
+        else tmem_dealloc(tmem_base, (uint32_t)g.tmem_cols);
+    }
 }
 
 }  // namespace tc
@@ -1329,10 +1454,25 @@ inline int sm_count() {
     return n;
 }
 
+// Which instantiations exist as CTA-pair kernels: every product with an MN-major N-side (the two
+// products with B, Gram, apply).  The fused pass stays on single CTAs: as pairs (leader loading the
+// R piece, peer the Q piece) it measured 1 - 1.5 ms slower per step at the 8B workload; its
+// epilogue waits on HBM, and two CTAs in lockstep have less slack for that than two free ones.
+constexpr bool pair_capable(int nmode, int epi, int xg) {
+    (void)epi; (void)xg;
+    return nmode == tc::N_IMG_MN;
+}
+
 template <int AMODE, int NMODE, int EPI, int XG>
 inline cudaError_t set_gemm_attr() {
-    return cudaFuncSetAttribute(tc::gemm_kernel<AMODE, NMODE, EPI, XG>,
-                                cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
+    cudaError_t e = cudaFuncSetAttribute(tc::gemm_kernel<AMODE, NMODE, EPI, XG, false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
+    if constexpr (pair_capable(NMODE, EPI, XG)) {
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc::gemm_kernel<AMODE, NMODE, EPI, XG, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
+    }
+    return e;
 }
 
 inline cudaError_t tensor_engine_set_attributes() {
@@ -1371,11 +1511,18 @@ inline void launch_pack(const Batch& b, Sel src, int64_t rows, int64_t cols, Img
 // Fills in the tiling, ring and tensor-memory fields and launches.
 template <int AMODE, int NMODE, int EPI, int XG>
 inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t st) {
+    if (g.fp16) { g.passes = 1; g.passes2 = 1; }
+    // CTA pairs need full 256-column instructions: every tile 256 or 512 columns wide.
+    bool pair = false;
+    if constexpr (pair_capable(NMODE, EPI, XG)) {
+        pair = g.BN % 256 == 0 && g.Ncols % g.BN == 0 && sm_count() >= 2;
+    }
+    g.pair = pair ? 1 : 0;
     g.m_tiles = (g.Mrows + tc::BM - 1) / tc::BM;
+    if (pair) g.m_tiles = (g.m_tiles + 1) / 2;      // scheduled row tiles of 256 rows
     g.n_tiles = (g.Ncols + g.BN - 1) / g.BN;
     g.k_blocks = (g.Kdim + tc::BK - 1) / tc::BK;
     g.total_tiles = b.count * g.m_tiles * g.n_tiles;
-    if (g.fp16) { g.passes = 1; g.passes2 = 1; }
     const int n1_terms = g.passes == 3 ? 2 : 1, n2_terms = g.passes2 == 3 ? 2 : 1;
     const int bn64 = (g.BN + 63) / 64 * 64;
     const int a_terms = (tc::a_is_buf(AMODE) || g.passes == 3 || (EPI == tc::EPI_K5 && g.passes2 == 3)) ? 2 : 1;
@@ -1389,8 +1536,14 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
         if (XG == 3 && a_terms == 1) g.epi_bufs = 1;
     }
     if (NMODE == tc::N_IMG_MN) {
-        g.ks = bn64 <= 128 ? 64 : (bn64 <= 256 ? 32 : 16);
-        g.n_piece_bytes = n1_terms * (bn64 / 64) * g.ks * 128;
+        if (pair) {
+            // each CTA holds half of the columns: same bytes per piece at twice the depth
+            g.ks = bn64 <= 256 ? 64 : 32;
+            g.n_piece_bytes = n1_terms * (bn64 / 128) * g.ks * 128;
+        } else {
+            g.ks = bn64 <= 128 ? 64 : (bn64 <= 256 ? 32 : 16);
+            g.n_piece_bytes = n1_terms * (bn64 / 64) * g.ks * 128;
+        }
     } else {
         g.ks = 64;
         g.n_piece_bytes = (n1_terms + (EPI == tc::EPI_K5 ? n2_terms : 0)) * tc::A_TERM_BYTES;
@@ -1408,13 +1561,29 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     const size_t smem = std::max<size_t>(fixed + (size_t)g.n_slots * g.n_piece_bytes, 120 * 1024);
     if (AMODE == tc::A_IMG_K) encode_img_map(&g.map_a, b, g.a, 128, 1, a_terms);
     else if (AMODE == tc::A_IMG_MN) encode_img_map(&g.map_a, b, g.a, 64, 2, a_terms);
-    if (NMODE == tc::N_IMG_MN) encode_img_map(&g.map_n1, b, g.n1, g.ks, bn64 / 64, n1_terms);
+    if (NMODE == tc::N_IMG_MN) encode_img_map(&g.map_n1, b, g.n1, g.ks, pair ? 2 : bn64 / 64, n1_terms);
     else encode_img_map(&g.map_n1, b, g.n1, 128, 1, n1_terms);
     if (EPI == tc::EPI_K5) encode_img_map(&g.map_n2, b, g.n2, 128, 1, n2_terms);
     if (engine_error()) return;
-    const int grid = std::min(g.total_tiles, sm_count());
     prof::Scope scope(stage, st);
-    tc::gemm_kernel<AMODE, NMODE, EPI, XG><<<grid, tc::gemm_threads(AMODE, EPI), smem, st>>>(b, g);
+    if constexpr (pair_capable(NMODE, EPI, XG)) {
+        if (pair) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)(2 * std::min(g.total_tiles, sm_count() / 2)), 1, 1);
+            cfg.blockDim = dim3((unsigned)tc::gemm_threads(AMODE, EPI), 1, 1);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, tc::gemm_kernel<AMODE, NMODE, EPI, XG, true>, b, g) != cudaSuccess)
+                engine_error() = 3;
+            return;
+        }
+    }
+    const int grid = std::min(g.total_tiles, sm_count());
+    tc::gemm_kernel<AMODE, NMODE, EPI, XG, false><<<grid, tc::gemm_threads(AMODE, EPI), smem, st>>>(b, g);
 }
 
 inline tc::Dest dest_none() {
