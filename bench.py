@@ -400,8 +400,12 @@ MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.32}
 
 
 def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):
-    """Same step, but every step copies all gradients host->device from pinned memory and all
-    updated weights device->host, inside the timed region."""
+    """Same step, end to end: every step copies all gradients host->device from pinned memory and
+    all updated weights device->host, inside the timed region.  The model is stepped in chunks of
+    consecutive matrices (one orthdion_step_grouped call per chunk) so that the copies of one chunk
+    overlap the kernels of another: an input stream, the compute stream and an output stream,
+    ordered by events (a chunk's gradients are not overwritten before its step has read them, its
+    weights not stepped again before they have been copied out)."""
     steps = max(1, min(args.steps, args.e2e_steps))
     g_host = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True) for g in Gsets[0]]
     x_host = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in Xs]
@@ -411,22 +415,66 @@ def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):
     h2d = sum(g.numel() * g.element_size() for g in g_host)
     d2h = sum(x.numel() * x.element_size() for x in x_host)
 
+    # chunks of consecutive matrices with about equal element counts
+    n_mat = len(Xs)
+    n_chunks = max(1, min(args.e2e_chunks, n_mat))
+    total = sum(x.numel() for x in Xs)
+    bounds, acc, nxt = [0], 0, 1
+    for i, x in enumerate(Xs):
+        acc += x.numel()
+        if nxt < n_chunks and acc >= total * nxt / n_chunks and i + 1 < n_mat:
+            bounds.append(i + 1)
+            nxt += 1
+    bounds.append(n_mat)
+    chunks = [range(bounds[k], bounds[k + 1]) for k in range(len(bounds) - 1) if bounds[k + 1] > bounds[k]]
+    t0 = tables[0]
+    hs_all = [t0.hs[i] for i in range(n_mat)]
+    Ms, Qs = t0._keep[1], t0._keep[3]
+    sub = [od.PointerTable([hs_all[i] for i in ch], [Xs[i] for i in ch], [Ms[i] for i in ch],
+                           [Gsets[0][i] for i in ch], [Qs[i] for i in ch]) for ch in chunks]
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    in_done = [torch.cuda.Event() for _ in chunks]
+    comp_done = [torch.cuda.Event() for _ in chunks]
+    out_done = [torch.cuda.Event() for _ in chunks]
+    first = [True]
+
     def one():
-        for gh, gd in zip(g_host, Gsets[0]):
-            gd.copy_(gh, non_blocking=True)
-        od.orthdion_step_grouped(tables[0], ws, stream)
-        for xh, xd in zip(x_host, Xs):
-            xh.copy_(xd, non_blocking=True)
+        for c, ch in enumerate(chunks):
+            with torch.cuda.stream(s_in):
+                if not first[0]:
+                    s_in.wait_event(comp_done[c])          # the previous step has read this chunk's G
+                for i in ch:
+                    Gsets[0][i].copy_(g_host[i], non_blocking=True)
+                in_done[c].record(s_in)
+            stream.wait_event(in_done[c])
+            if not first[0]:
+                stream.wait_event(out_done[c])             # the previous X of this chunk has left
+            od.orthdion_step_grouped(sub[c], ws, stream)
+            comp_done[c].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(comp_done[c])
+                for i in ch:
+                    x_host[i].copy_(Xs[i], non_blocking=True)
+                out_done[c].record(s_out)
+        first[0] = False
+
+    def join():
+        stream.wait_stream(s_in)
+        stream.wait_stream(s_out)
 
     one()
+    join()
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     ev0.record(stream)
+    s_in.wait_event(ev0)
+    s_out.wait_event(ev0)
     for _ in range(steps):
         one()
+    join()
     ev1.record(stream)
     torch.cuda.synchronize()
     ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
@@ -437,7 +485,8 @@ def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):
         dist.all_reduce(t)
         job_elements = float(t.item())
     return {"value": job_elements / (ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": ms_step, "steps": steps}
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms_step, "steps": steps,
+            "pipeline": f"{len(chunks)} chunks of consecutive matrices, copies on their own streams"}
 
 
 def main():
@@ -459,6 +508,8 @@ def main():
                     help="on-device diagnostics inside the timed step (0 off, 1 factor diagnostics, 3 plus buffer norms)")
     ap.add_argument("--grad-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-chunks", type=int, default=8,
+                    help="grouped calls per end-to-end step (copies of one chunk overlap the kernels of another)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")

@@ -103,7 +103,10 @@ def test_cfg0_chained_both_modes(engine):
 # ------------------------------------------------------------------ one step, several shapes
 SHAPES_ANY = [(200, 328, 24), (129, 520, 8), (64, 64, 64), (520, 136, 40), (96, 1000, 1), (300, 77, 5)]
 SHAPES_TENSOR = [(256, 512, 16), (384, 640, 64), (200, 328, 48), (1000, 264, 128), (136, 2056, 32),
-                 (640, 384, 272), (64, 64, 64), (96, 1000, 16), (48, 136, 16), (16, 16, 16)]
+                 (640, 384, 272), (64, 64, 64), (96, 1000, 16), (48, 136, 16), (16, 16, 16),
+                 # ranks that are multiples of 256 run as CTA pairs: odd and even numbers of 128-row
+                 # tiles on either side, a ragged last tile, two 512-column tiles (r = 1024)
+                 (384, 640, 256), (1000, 1032, 256), (1152, 768, 512), (1300, 1024, 1024)]
 
 
 @pytest.mark.parametrize("shape", SHAPES_ANY)
