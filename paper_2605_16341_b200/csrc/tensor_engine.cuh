@@ -642,18 +642,19 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             const TileCoord c = decode_tile<EPI>(batch, g, t, scache, crank);
             if (!c.active) continue;
             if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+            // orders this tile's MMAs after the epilogue's tensor-memory loads.  (The operand waits
+            // below need no tcgen05 fence: the operands arrive through the async proxy or behind
+            // a proxy fence, and a fence per piece stalled the issuer for hundreds of cycles.)
             tc_fence_after();
             const uint32_t dacc = tmem_base + acc * acc_stride;
             for (int kb = 0; kb < c.kb_end && ok; ++kb) {
                 if (!mbar_wait(a_full0 + 8 * as, aph, abort_flag)) { ok = false; break; }
-                tc_fence_after();
                 const uint64_t a_kb = a_hi + (a_ring16 + as * a_slot16);
                 if (NMODE == N_IMG_MN) {
                     const int pieces = mn_pieces(g, kb);
                     const int per_piece = g.ks / 16;
                     for (int sub = 0; sub < pieces && ok; ++sub) {
                         if (!mbar_wait(n_full0 + 8 * ns, nph, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
                         if (lane == 0) {
                             const uint64_t n_pc = n_hi + (n_ring16 + ns * n_slot16);
                             const int k0 = kb * BK + sub * g.ks;
@@ -684,7 +685,6 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                     for (int ch = 0; ch < chunks && ok; ++ch) {
                         if (!k_piece_active(g, c, kb, ch)) continue;
                         if (!mbar_wait(n_full0 + 8 * ns, nph, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
                         if (lane == 0) {
                             const uint32_t sa = smem_u32(a_ring + as * g.a_slot_bytes);
                             const uint32_t sn = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
@@ -698,10 +698,21 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                             // the P slice from shared memory once.
                             const bool both = EPI == EPI_K5 && g.passes == 1 && g.passes2 == 1 && ncols == 128 && g.BN == 128;
                             const uint32_t idesc2 = instr_desc(256u, A_MN ? 1u : 0u, 0u, fmt, MROWS);
-                            // (Descriptors are rebuilt per instruction here on purpose: with the additive
-                            // form of the other branch the fused pass measured 38 ms instead of 26 ms per
-                            // step; its N = 128 instructions run best when they are not issued back to back.)
-                            for (int j = 0; j < nsl; ++j) {
+                            if (both) {
+                                // one instruction per 16-deep slice; descriptors advanced by additions so
+                                // that the issuing thread spends a handful of operations per instruction
+                                uint64_t a0 = a_hi + (a_ring16 + as * a_slot16);
+                                uint64_t b0 = n_hi + (n_ring16 + ns * n_slot16);
+                                const uint32_t d1 = dacc + ch * 128;
+                                umma_any<PAIR>(d1, a0, b0, idesc2, kb > 0 ? 1u : 0u);
+                                for (int j = 1; j < nsl; ++j) {
+                                    a0 += a_slice16; b0 += n_slice16;
+                                    umma_any<PAIR>(d1, a0, b0, idesc2, 1u);
+                                }
+                            }
+                            // (In the general form below the descriptors are rebuilt per instruction on
+                            // purpose: its N = 128 instructions ran best when not issued back to back.)
+                            for (int j = 0; j < nsl && !both; ++j) {
                                 const uint64_t a0 = A_MN ? smem_desc(sa + j * 2048, 8192, 1024)
                                                          : smem_desc(sa + j * 32, 16, 1024);
                                 const uint64_t a1 = A_MN ? smem_desc(sa + A_TERM_BYTES + j * 2048, 8192, 1024)
@@ -710,7 +721,6 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                 const uint64_t b1 = smem_desc(sn + A_TERM_BYTES + j * 32, 16, 1024);
                                 const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
                                 const uint32_t d1 = dacc + ch * 128;
-                                if (both) { umma_any<PAIR>(d1, a0, b0, idesc2, accum); continue; }
                                 umma_any<PAIR>(d1, a0, b0, idesc, accum);
                                 if (g.passes == 3) {
                                     umma_any<PAIR>(d1, a0, b1, idesc, 1u);
