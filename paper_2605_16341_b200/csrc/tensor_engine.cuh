@@ -587,11 +587,17 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                     const uint32_t dst = smem_u32(n_ring + (size_t)ns * g.n_piece_bytes);
                     if (PAIR) {
                         // this CTA's half of the N-side: per 256-column block its two 64-column groups
+                        // (MN-major), or the R piece (leader) / the Q piece (peer) of the fused pass
                         mbar_arrive_expect_tx_remote(fb, (uint32_t)g.n_piece_bytes);
-                        const uint32_t blk_bytes = (uint32_t)n1_terms * 2u * group_stride;
-                        for (int blk = 0; blk * 256 < nc.bn; ++blk)
-                            tma_load_box_pair(dst + blk * blk_bytes, &g.map_n1, nkb * BK + npc * g.ks,
-                                              nc.n0 / 64 + blk * 4 + crank * 2, plane, nc.b, fb);
+                        if (NMODE == N_IMG_MN) {
+                            const uint32_t blk_bytes = (uint32_t)n1_terms * 2u * group_stride;
+                            for (int blk = 0; blk * 256 < nc.bn; ++blk)
+                                tma_load_box_pair(dst + blk * blk_bytes, &g.map_n1, nkb * BK + npc * g.ks,
+                                                  nc.n0 / 64 + blk * 4 + crank * 2, plane, nc.b, fb);
+                        } else {
+                            tma_load_box_pair(dst, crank == 0 ? &g.map_n1 : &g.map_n2, nc.n0 + npc * 128, nkb, plane,
+                                              nc.b, fb);
+                        }
                     } else {
                         mbar_arrive_expect_tx(fb, (uint32_t)g.n_piece_bytes);
                         if (NMODE == N_IMG_MN) {
@@ -1465,12 +1471,10 @@ inline int sm_count() {
 }
 
 // Which instantiations exist as CTA-pair kernels: every product with an MN-major N-side (the two
-// products with B, Gram, apply).  The fused pass stays on single CTAs: as pairs (leader loading the
-// R piece, peer the Q piece) it measured 1 - 1.5 ms slower per step at the 8B workload; its
-// epilogue waits on HBM, and two CTAs in lockstep have less slack for that than two free ones.
+// products with B, Gram, apply) and the fused pass on bf16 G and X in its single-term form, where
+// the leader loads the R pieces and the peer the Q pieces (operand bytes per element 24 -> 16).
 constexpr bool pair_capable(int nmode, int epi, int xg) {
-    (void)epi; (void)xg;
-    return nmode == tc::N_IMG_MN;
+    return nmode == tc::N_IMG_MN || (epi == tc::EPI_K5 && xg == 3);
 }
 
 template <int AMODE, int NMODE, int EPI, int XG>
@@ -1522,10 +1526,13 @@ inline void launch_pack(const Batch& b, Sel src, int64_t rows, int64_t cols, Img
 template <int AMODE, int NMODE, int EPI, int XG>
 inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t st) {
     if (g.fp16) { g.passes = 1; g.passes2 = 1; }
-    // CTA pairs need full 256-column instructions: every tile 256 or 512 columns wide.
+    // CTA pairs need full 256-column instructions: every tile 256 or 512 columns wide (MN-major
+    // N-side), or the fused pass in its single-term form with full 128-column tiles.
     bool pair = false;
     if constexpr (pair_capable(NMODE, EPI, XG)) {
-        pair = g.BN % 256 == 0 && g.Ncols % g.BN == 0 && sm_count() >= 2;
+        if (NMODE == tc::N_IMG_MN) pair = g.BN % 256 == 0 && g.Ncols % g.BN == 0;
+        else pair = g.passes == 1 && g.passes2 == 1 && g.BN == 128 && g.Ncols % 128 == 0;
+        if (sm_count() < 2) pair = false;
     }
     g.pair = pair ? 1 : 0;
     g.m_tiles = (g.Mrows + tc::BM - 1) / tc::BM;
@@ -1557,6 +1564,7 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     } else {
         g.ks = 64;
         g.n_piece_bytes = (n1_terms + (EPI == tc::EPI_K5 ? n2_terms : 0)) * tc::A_TERM_BYTES;
+        if (pair) g.n_piece_bytes = tc::A_TERM_BYTES;    // the R piece (leader) or the Q piece (peer)
     }
     const int accw = (EPI == tc::EPI_K5) ? 2 * g.BN : g.BN;
     g.acc_bufs = (2 * accw <= 512) ? 2 : 1;
