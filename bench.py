@@ -394,9 +394,9 @@ def run_ours(args):
 
 
 # DRAM bytes per parameter element of a stage, measured with ncu on a smaller case of the same
-# kernel (profiles/fused_feedback_update_kernel_cfg4_4layers.md: 6.740 GB over 469.8 M elements);
+# kernel (profiles/fused_feedback_update_kernel_cfg4_4layers.md: 6.782 GB over 469.8 M elements);
 # traffic grows in proportion to the elements, so a step's traffic is this figure x its elements.
-MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.35}
+MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.43}
 
 
 def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):

@@ -11,8 +11,8 @@
 // the current chunk is multiplied, so the L2 latency hides behind the work.
 //
 // Right-looking Cholesky with 32-wide panels:
-//   diagonal block   one warp, rows in registers, pivots and columns passed by shuffles; its
-//                    inverse (needed at the end anyway) replaces it in place right away
+//   diagonal block   in shared memory: columns scaled by one warp, rank-one updates by all
+//                    threads; then one warp inverts it (needed at the end anyway) in place
 //   panel            rows below  <-  rows below * inv(L_kk)^T          (tile products, depth 32)
 //   trailing update  W22 -= L21 L21^T, lower tiles only                (tile products, depth 32)
 // then the inverse of the factor by combining diagonal blocks pairwise (32, 64, 128, ...):
@@ -201,34 +201,12 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
     __syncthreads();
 }
 
-// One warp: Cholesky of a 32 x 32 block held one row per lane (a[c], c <= lane; rows >= nb must be
-// identity rows).  On return a[] is the row of L.  Returns true if a pivot was not positive.
-__device__ __forceinline__ bool warp_chol32(float (&a)[32], int lane, int nb, float& dmin, float& dmax) {
-    bool fail = false;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        float d = __shfl_sync(0xffffffffu, a[j], j);
-        if (!(d > 0.f) || !(d <= 3.0e38f)) { if (j < nb) fail = true; d = 1.f; }
-        const float s = sqrtf(d);
-        if (j < nb) { dmin = fminf(dmin, s); dmax = fmaxf(dmax, s); }
-        const float lij = (lane > j) ? a[j] / s : 0.f;
-        if (lane == j) a[j] = s;
-        else if (lane > j) a[j] = lij;
-#pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            if (c > j) {      // both loops run over the full range so that every index is a constant
-                const float lcj = __shfl_sync(0xffffffffu, lij, c);
-                if (lane >= c) a[c] = fmaf(-lij, lcj, a[c]);
-            }
-        }
-    }
-    return fail;
-}
-
 __global__ void __launch_bounds__(CT_THREADS, 2)
 chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     __shared__ __align__(16) __nv_bfloat16 s_stage[4 * 64 * CT_LDK];
     __shared__ TcTask s_tasks[CT_MAX_TASKS];
+    __shared__ float s_blk[32 * 33];
+    __shared__ float s_piv[32];
     __shared__ float s_diag[1024];
     __shared__ float s_rowsum[1024];
     __shared__ float red[8];
@@ -354,50 +332,84 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     for (int attempt = 0; attempt < max_attempts && !ok; ++attempt) {
         const float shift = attempt ? a.shift_rel * trace : 0.f;
         // W <- lower(A) + shift*I (diagonal from s_diag), strict upper part zero; 4 columns per thread
+        // (eight loads in flight per thread: one at a time, the L2 round trips of this copy alone
+        // were 8 % of the kernel)
         const int r4 = r / 4;
-        for (int q = tid; q < r * r4; q += CT_THREADS) {
-            const int i = q / r4, j4 = (q - i * r4) * 4;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (j4 <= i) {
-                v = *reinterpret_cast<const float4*>(A + i * r + j4);
-                if (j4 + 0 > i) v.x = 0.f; else if (j4 + 0 == i) v.x = s_diag[i] + shift;
-                if (j4 + 1 > i) v.y = 0.f; else if (j4 + 1 == i) v.y = s_diag[i] + shift;
-                if (j4 + 2 > i) v.z = 0.f; else if (j4 + 2 == i) v.z = s_diag[i] + shift;
-                if (j4 + 3 > i) v.w = 0.f; else if (j4 + 3 == i) v.w = s_diag[i] + shift;
+        for (int q0 = tid; q0 < r * r4; q0 += 8 * CT_THREADS) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + u * CT_THREADS;
+                const int i = q / r4, j4 = (q - i * r4) * 4;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q < r * r4 && j4 <= i) v[u] = *reinterpret_cast<const float4*>(A + i * r + j4);
             }
-            *reinterpret_cast<float4*>(W + i * r + j4) = v;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + u * CT_THREADS;
+                if (q >= r * r4) break;
+                const int i = q / r4, j4 = (q - i * r4) * 4;
+                if (j4 <= i) {
+                    if (j4 + 0 > i) v[u].x = 0.f; else if (j4 + 0 == i) v[u].x = s_diag[i] + shift;
+                    if (j4 + 1 > i) v[u].y = 0.f; else if (j4 + 1 == i) v[u].y = s_diag[i] + shift;
+                    if (j4 + 2 > i) v[u].z = 0.f; else if (j4 + 2 == i) v[u].z = s_diag[i] + shift;
+                    if (j4 + 3 > i) v[u].w = 0.f; else if (j4 + 3 == i) v[u].w = s_diag[i] + shift;
+                }
+                *reinterpret_cast<float4*>(W + i * r + j4) = v[u];
+            }
         }
         if (tid == 0) { s_fail = 0; s_dmin = 3.0e38f; s_dmax = 0.f; }
         __syncthreads();
 
         for (int k0 = 0; k0 < r; k0 += CT_NB) {
             const int nb = min(CT_NB, r - k0);
-            if (warp == 0) {
-                // factor the diagonal block and replace it by its inverse
-                float row[32];
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                    row[c] = (lane < nb && c <= lane) ? W[(k0 + lane) * r + k0 + c] : (c == lane ? 1.f : 0.f);
-                float dmin = 3.0e38f, dmax = 0.f;
-                const bool fail = warp_chol32(row, lane, nb, dmin, dmax);
-                // lane c solves L x = e_c (column c of the inverse); L(i, p) comes from lane i's registers
-                float x[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float sacc = (i == lane) ? 1.f : 0.f;
-#pragma unroll
-                    for (int p = 0; p < 32; ++p)
-                        if (p < i) sacc = fmaf(-__shfl_sync(0xffffffffu, row[p], i), x[p], sacc);
-                    const float lii = __shfl_sync(0xffffffffu, row[i], i);
-                    x[i] = (i >= lane) ? sacc / lii : 0.f;
+            // Diagonal block: factored in shared memory by all threads (column scaling by one warp,
+            // rank-one update by everybody, two barriers per column), then inverted by one warp
+            // (thread c solves L x = e_c with x in registers; L(i, p) are broadcast reads).  The
+            // inverse replaces the block in place right away: it is needed at the end anyway.
+            {
+                for (int e = tid; e < 1024; e += CT_THREADS) {
+                    const int i = e >> 5, c = e & 31;
+                    float v = (i == c) ? 1.f : 0.f;          // rows beyond nb are identity rows
+                    if (i < nb && c <= i) v = W[(k0 + i) * r + k0 + c];
+                    s_blk[i * 33 + c] = v;
                 }
+                __syncthreads();
+                bool fail = false;
+                float dmin = 3.0e38f, dmax = 0.f;             // every thread tracks the same values
+                for (int j = 0; j < 32; ++j) {
+                    float d = s_blk[j * 33 + j];
+                    if (!(d > 0.f) || !(d <= 3.0e38f)) { if (j < nb) fail = true; d = 1.f; }
+                    const float sq = sqrtf(d);
+                    if (j < nb) { dmin = fminf(dmin, sq); dmax = fmaxf(dmax, sq); }
+                    if (tid == j) s_piv[j] = sq;
+                    else if (tid > j && tid < 32) s_blk[tid * 33 + j] = s_blk[tid * 33 + j] / sq;
+                    __syncthreads();
+                    for (int e = tid; e < 1024; e += CT_THREADS) {
+                        const int i = e >> 5, c = e & 31;
+                        if (c > j && i >= c)
+                            s_blk[i * 33 + c] = fmaf(-s_blk[i * 33 + j], s_blk[c * 33 + j], s_blk[i * 33 + c]);
+                    }
+                    __syncthreads();
+                }
+                if (warp == 0) {
+                    float x[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (i < nb && lane < nb && i >= lane) W[(k0 + i) * r + k0 + lane] = x[i];
-                if (lane == 0) {
-                    if (fail) s_fail = 1;
-                    s_dmin = fminf(s_dmin, dmin);
-                    s_dmax = fmaxf(s_dmax, dmax);
+                    for (int i = 0; i < 32; ++i) {
+                        float sacc = (i == lane) ? 1.f : 0.f;
+#pragma unroll
+                        for (int p = 0; p < 32; ++p)
+                            if (p < i) sacc = fmaf(-s_blk[i * 33 + p], x[p], sacc);
+                        x[i] = (i >= lane) ? sacc / s_piv[i] : 0.f;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < nb && lane < nb && i >= lane) W[(k0 + i) * r + k0 + lane] = x[i];
+                    if (lane == 0) {
+                        if (fail) s_fail = 1;
+                        s_dmin = fminf(s_dmin, dmin);
+                        s_dmax = fmaxf(s_dmax, dmax);
+                    }
                 }
             }
             __syncthreads();
@@ -495,18 +507,30 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         unsigned char* __restrict__ scr = reinterpret_cast<unsigned char*>(w.scratch);
         const float* __restrict__ Wr = W;
         const int chunks = a.img.panels * a.img.rows_pad * 8;
-        for (int q = tid; q < chunks; q += CT_THREADS) {
-            // consecutive threads take consecutive image rows (consecutive k: contiguous in W)
-            const int row = q % a.img.rows_pad, c = (q / a.img.rows_pad) % 8, panel = q / (8 * a.img.rows_pad);
-            const int col = panel * 64 + c * 8;
-            float v[8];
+        for (int q0 = tid; q0 < chunks; q0 += 4 * CT_THREADS) {
+            // consecutive threads take consecutive image rows (consecutive k: contiguous in W);
+            // four chunks (32 loads) in flight per thread
+            float v[4][8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = (row < r && col + i < r) ? Wr[(col + i) * r + row] : 0.f;
-            uint4 t0, t1;
-            split8(v, t0, t1);
-            const int o = img_chunk_offset(row, c);
-            *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 0, panel, row) + o) = t0;
-            *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 1, panel, row) + o) = t1;
+            for (int u = 0; u < 4; ++u) {
+                const int q = q0 + u * CT_THREADS;
+                const int row = q % a.img.rows_pad, c = (q / a.img.rows_pad) % 8, panel = q / (8 * a.img.rows_pad);
+                const int col = panel * 64 + c * 8;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    v[u][i] = (q < chunks && row < r && col + i < r) ? Wr[(col + i) * r + row] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int q = q0 + u * CT_THREADS;
+                if (q >= chunks) break;
+                const int row = q % a.img.rows_pad, c = (q / a.img.rows_pad) % 8, panel = q / (8 * a.img.rows_pad);
+                uint4 t0, t1;
+                split8(v[u], t0, t1);
+                const int o = img_chunk_offset(row, c);
+                *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 0, panel, row) + o) = t0;
+                *reinterpret_cast<uint4*>(scr + img_row_offset(a.img, 1, panel, row) + o) = t1;
+            }
         }
     }
 }
