@@ -72,15 +72,21 @@ def stage_models(matrices, mode_orth=True):
         xb = 2 if s.x_dtype == torch.bfloat16 else 4
         add("k1_buffer_times_q", 2.0 * m * n * r, (4 + gb) * m * n + 4.0 * (n + m) * r)
         add("k3_buffer_t_times_p", 2.0 * m * n * r, (4 + gb) * m * n + 4.0 * (n + m) * r)
-        # factor reads of the fused pass: fp16 planes of P, R, Q for bf16 weights, two bf16 terms else
-        fb = 2.0 if s.x_dtype == torch.bfloat16 else 4.0
-        add("k5_feedback_update", 4.0 * m * n * r, (8 + gb + 2 * xb) * m * n + fb * (2 * n + m) * r)
+        # the fused pass: M read and written, G read, X read and written (14 B per element with
+        # bf16 X and G); the operand planes of P, R, Q it also reads are reported on their own
+        add("k5_feedback_update", 4.0 * m * n * r, (8 + gb + 2 * xb) * m * n)
         qrs = [m] + ([n] if mode_orth else [])
         for k in qrs:
             add("gram", 2 * 2.0 * k * r * r, 2 * 4.0 * k * r)
             add("apply_inverse", 2 * 1.0 * k * r * r, 2 * 12.0 * k * r)
             add("cholesky_inverse", 2 * 2.0 * r ** 3 / 3.0, 2 * 8.0 * r * r)
     return out
+
+
+def k5_factor_plane_bytes(matrices):
+    """Bytes of the operand planes of P, R, Q that the fused pass reads once from HBM (fp16 planes
+    for bf16 weights, two bf16 terms otherwise); not part of its 14 B per element."""
+    return sum((2.0 if s.x_dtype == torch.bfloat16 else 4.0) * (2 * s.n + s.m) * s.r for s in matrices)
 
 
 class ClockSampler:
@@ -169,6 +175,34 @@ def cpu_oracle_sample(w, steps=1, warmup=0):
     return spec.numel / sec, sec, desc
 
 
+def cpu_oracle_per_class(w, mode_orth=True):
+    """One oracle step of the first matrix of every distinct shape of the workload, timed on the
+    host cores, and the whole-model step extrapolated from the class counts:
+    seconds(model) = sum over classes of (matrices in the class) x (seconds of its sample).
+    Returns (elements/s, seconds, description, per-class list)."""
+    from oracle import orthdion_oracle as orc
+    classes = wl.shape_classes(w.matrices)
+    per, total = [], 0.0
+    for key, members in classes.items():
+        idx = members[0]
+        spec = w.matrices[idx]
+        X, M, Q = wl.initial_state(spec, 0, idx)
+        basis = wl.grad_basis(w, spec, 0, idx)
+        G = wl.gradient(w, spec, 0, idx, 0, basis).double().numpy()
+        Xo, Mo, Qo = X.double().numpy(), M.double().numpy(), Q.double().numpy()
+        del X, M, Q, basis
+        t0 = time.perf_counter()
+        orc.step(Xo, Mo, G, Qo, eta=w.eta, mu=w.mu, wd=w.wd, mode=orc.ORTH if mode_orth else orc.COLNORM)
+        dt = time.perf_counter() - t0
+        del Xo, Mo, Qo, G
+        per.append({"shape": f"{spec.m}x{spec.n}", "r": spec.r, "matrices": len(members), "seconds": dt})
+        total += dt * len(members)
+    desc = (f"extrapolated: one float64 numpy oracle step of one matrix per distinct shape of {w.name} "
+            f"({', '.join(p['shape'] for p in per)}; {sum(p['seconds'] for p in per):.1f} s of CPU work), "
+            f"model step = sum over shapes of count x seconds; elements/s = all elements / that")
+    return w.numel / total, total, desc, per
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -186,10 +220,10 @@ def run_reference(args):
         return
     w = wl.workload(args.workload, layers=args.layers)
     steps = max(1, args.steps)
-    val, sec, desc = cpu_oracle_sample(w, steps=steps, warmup=min(args.warmup, 1))
+    val, sec, desc = cpu_oracle_sample(w, steps=steps, warmup=max(0, args.warmup))
     cores = blas_threads()
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3,
+            "steps": steps, "warmup": max(0, args.warmup), "ms_per_step": sec * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": w.name, "sample": desc},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
@@ -215,6 +249,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     w = wl.workload(args.workload, layers=args.layers, r=args.rank)
+    if args.lanes:
+        od.orthdion_set_concurrency(args.lanes)
     mode = od.MODE_ORTH if args.mode == "orth" else od.MODE_COLNORM
     seed = 1000 + rank
     all_matrices = w.matrices
@@ -356,15 +392,18 @@ def run_ours(args):
         roofline.update({"kernel": dominant, "launches_per_step": stages[dominant]["launches_per_step"],
                          "per": "step (sum over the launches of this kernel in one step)",
                          "algorithmic": (b if roofline["bound"] == "hbm" else f),
+                         "algorithmic_per_element": ((b / w.numel) if roofline["bound"] == "hbm" else None),
+                         "factor_plane_bytes": (k5_factor_plane_bytes(w.matrices)
+                                                if dominant == "k5_feedback_update" else None),
                          "traffic": (bpe * w.numel if (bpe and args.mode == "orth" and not args.passes) else None),
                          "peak_source": peaks["source"] + (" (sustained bf16 figure: kernel timed inside a long step)"
                                                            if roofline["bound"] == "tensor" else "")})
 
     cpu = None
     if not args.no_cpu_baseline:
-        val, sec, desc = cpu_oracle_sample(w, steps=1)
+        val, sec, desc, per = cpu_oracle_per_class(w, orth)
         cpu = {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc,
-               "seconds": sec}
+               "seconds_per_model_step_extrapolated": sec, "per_shape": per}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -393,9 +432,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes per parameter element of a stage, measured with ncu on a smaller case of the same
-# kernel (profiles/fused_feedback_update_kernel_cfg4_4layers.md: 6.782 GB over 469.8 M elements);
-# traffic grows in proportion to the elements, so a step's traffic is this figure x its elements.
+# DRAM bytes per parameter element of a stage, measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum of one launch) on a 4-layer case of the same kernel: 6.782 GB over
+# 469.8 M elements.  Traffic grows in proportion to the elements, so a step's traffic is this
+# figure x its elements.  Set to None whenever the kernel changes until the counters are retaken.
 MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.43}
 
 
@@ -506,8 +546,10 @@ def main():
                     help="bf16 split passes of the four product groups, e.g. 3,3,3,1 (0 keeps the default)")
     ap.add_argument("--diagnostics", type=int, default=0, choices=[0, 1, 3],
                     help="on-device diagnostics inside the timed step (0 off, 1 factor diagnostics, 3 plus buffer norms)")
+    ap.add_argument("--lanes", type=int, default=None,
+                    help="internal streams a grouped call spreads its launch batches over (library default if unset)")
     ap.add_argument("--grad-sets", type=int, default=2)
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--e2e-chunks", type=int, default=8,
                     help="grouped calls per end-to-end step (copies of one chunk overlap the kernels of another)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -516,8 +558,31 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
     else:
         run_ours(args)
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this same command line under
+    torch.distributed.run on this node (one process per GPU, rendezvous on 127.0.0.1) and pass
+    their output through.  NCCL's own initialisation lines go to stderr."""
+    import socket
+    have = torch.cuda.device_count()
+    if have < n:
+        print(f"bench.py: --gpus {n} asked for, {have} CUDA device(s) visible", file=sys.stderr)
+        return 2
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd, env=env)
 
 
 if __name__ == "__main__":

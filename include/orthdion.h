@@ -1,21 +1,24 @@
 /* orthdion.h - C interface of the B200 (sm_100a) Orth-Dion / Dion optimizer-step library.
  *
- * One call of orthdion_step performs, for one weight matrix, the step of Algorithm 1 of the
- * paper ("Orth-Dion / Stripped Dion (one step)"; appendix algorithms "Stripped Dion" and
- * "Orth-Dion"), written with the letters of this interface:
+ * One call of orthdion_step advances one weight matrix by one step of the paper's Algorithm 1
+ * (the one-step statement of Orth-Dion and of Dion with its auxiliary machinery stripped; the
+ * appendix gives both as full loops).  The library runs it as five stages, written here with the
+ * letters of this interface (the paper's letters in brackets):
  *
- *     B  = M + G                                 buffer            (Alg. 1, buffer step)
- *     P  = orth(B * Q_prev)                      left factor       (Alg. 1, left-factor step)
- *     R  = B^T * P                               right factor      (Alg. 1, right-factor step)
- *     Q  = orth(R)   [ORTH]   |  ColNorm(R) [COLNORM]              (Alg. 1, normalisation step)
- *     X <- (1 - eta*wd) * X - eta*scale * P * Q^T                  (Alg. 1, update step)
- *     M <- a * B - b * P * R^T                   error feedback    (Alg. 1, error-feedback step)
- *     Q_prev <- Q                                warm start        (Alg. 1, warm-start step)
+ *   K1     Y = (M + G) * Q_prev        the buffer B = M + G [M_t = G_t + R_t] is formed on the
+ *                                      fly and never stored; Q_prev is the carried right
+ *                                      factor [V_{t-1}]
+ *   QR     P = orth(Y)                 left factor [U_t]
+ *   K3     R = (M + G)^T * P           un-normalised right factor [W_t]
+ *   QR or  Q = orth(R)   (ORTH)        Orth-Dion's normalisation of the right factor, or
+ *   scale  Q = ColNorm(R) (COLNORM)    Dion's unit-length columns [V_t]
+ *   K5     X <- (1 - eta*wd) * X - eta*scale * P * Q^T      weight update, and in the same pass
+ *          M <- a * (M + G) - b * P * R^T                   the error-feedback residual [R_{t+1}]
  *
- * Paper letters: G_t = G, R_t = M (residual), M_t = B, V_{t-1} = Q_prev, U_t = P, W_t = R.
- * orth(.) is the thin QR factor with a positive diagonal in the triangular factor
- * (CholeskyQR2 on the device, with a shifted third pass when the Gram matrix is
- * ill-conditioned).  (a, b) default to (1, 1 - mu); the paper's error-feedback step is (beta, beta).
+ * Q then serves as Q_prev of the next step.  orth(.) is the thin QR factor with a positive
+ * diagonal in the triangular factor (CholeskyQR2 on the device, with a shifted third pass when
+ * the Gram matrix is ill-conditioned).  (a, b) default to (1, 1 - mu); the paper's own residual
+ * rule is (beta, beta).
  *
  * Conventions
  *  - Every matrix pointer is a DEVICE pointer owned by the caller; matrices are row-major and
@@ -77,7 +80,9 @@ typedef struct orthdion_plan* orthdion_t;
 #define ORTHDION_STATUS_RANK_DEFICIENT  4   /* factorisation failed: X, M, Q left unchanged     */
 #define ORTHDION_STATUS_NONFINITE       8   /* a Gram matrix held Inf/NaN: treated as failure   */
 #define ORTHDION_STATUS_ZERO_COLUMN    16   /* COLNORM met a zero column of R (kept zero)       */
-#define ORTHDION_STATUS_WAIT_LIMIT     32   /* a bounded device-side wait expired (kernel bug)  */
+#define ORTHDION_STATUS_WAIT_LIMIT     32   /* a bounded device-side wait expired (kernel bug): */
+                                            /* set on every matrix of the launch; M and X of    */
+                                            /* those matrices may be partially updated          */
 
 /* Create a plan for m x n matrices at rank r (inputs of Algorithm 1: step size eta, EF
  * coefficient; mu gives the default (a, b) = (1, 1 - mu)).  Defaults: X and G bfloat16,
@@ -112,12 +117,22 @@ int orthdion_step(orthdion_t h, void* X, float* M, const void* G, float* Q,
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /* One step for `count` matrices; hs[i] is the plan of matrix i.  X, M, G, Q are HOST arrays of
- * `count` device pointers.  Matrices are packed by equal plan parameters ("sort-and-pack"
- * batching, appendix on the wide-model study) and every stage runs once per pack.  Results per
- * matrix are identical to orthdion_step. */
+ * `count` device pointers.  Matrices with equal plan parameters are sorted into packs and every
+ * stage runs once per pack (the batching of equal shapes that the paper's appendix on its
+ * wide-model study mentions).  Results per matrix are identical to orthdion_step. */
 int orthdion_step_grouped(const orthdion_t* hs, int32_t count,
                           void* const* X, float* const* M, const void* const* G, float* const* Q,
                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* How many launch batches (matrices of equal plan) a grouped call may step side by side.  The
+ * optimizer steps of two matrices are independent (nothing in Algorithm 1 couples them), so the
+ * grouped call forks the caller's stream into `lanes` internal streams, runs every batch's
+ * stage sequence on one of them and joins them again before it returns: everything enqueued on
+ * `stream` after the call still waits for the whole step, and the host never blocks.  Results per
+ * matrix are bit for bit those of lanes = 1.  1 <= lanes <= 8; default 4.  Process-wide; the first
+ * grouped call on a device creates that device's internal streams and events (no device memory);
+ * two grouped calls on the same device are serialised on the host while they enqueue. */
+int orthdion_set_concurrency(int32_t lanes);
 
 /* One step for one matrix without any caller-provided workspace and without any device-memory
  * allocation.  (The paper has no counterpart: this entry point exists for the integration, not
@@ -191,8 +206,9 @@ int orthdion_last_diagnostics(const orthdion_t* hs, int32_t count, void* workspa
 int orthdion_rank_policy(double e_t, int32_t r_t, double ema_prev, int32_t r_min, int32_t r_max,
                          double alpha, double gamma, int32_t multiple, double* ema_out, int32_t* r_next);
 
-/* "Resize U, V to rank r_{t+1} (truncate or pad)" for the one factor that is carried between
- * steps: Q_new (n x r_new, device, row-major) receives the leading min(r_old, r_new) columns of
+/* The resize step of the rank-selection algorithm, for the one factor that is carried between
+ * steps (the left factor is recomputed by every step): the warm-start factor is cut down or
+ * extended to the new rank.  Q_new (n x r_new, device, row-major) receives the leading min(r_old, r_new) columns of
  * Q_old (n x r_old) and, when r_new > r_old, the columns of `pad` (n x (r_new - r_old), device,
  * row-major; may be null otherwise).  The paper does not say what the new columns hold: the caller
  * supplies them (any columns that keep B*Q of full column rank serve the power iteration, e.g.

@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
     L.orthdion_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.orthdion_get_factors.argtypes = [pvp, i32, i32, vp, pvp, pvp]
     L.orthdion_last_status.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(i32)]
+    L.orthdion_set_concurrency.argtypes = [i32]
     L.orthdion_set_diagnostics.argtypes = [vp, i32]
     L.orthdion_last_diagnostics.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(ctypes.c_float)]
     dbl = ctypes.c_double
@@ -94,7 +95,7 @@ def lib() -> ctypes.CDLL:
     L.orthdion_stage_name.restype = ctypes.c_char_p
     for name in ("create", "destroy", "set_dtypes", "set_lr", "set_scale", "set_ef", "set_engine",
                  "set_passes", "step", "step_grouped", "step_noalloc", "get_factors", "last_status",
-                 "set_diagnostics", "last_diagnostics", "rank_policy", "resize_factor"):
+                 "set_diagnostics", "last_diagnostics", "rank_policy", "resize_factor", "set_concurrency"):
         getattr(L, "orthdion_" + name).restype = i32
     _lib = L
     return L
@@ -104,7 +105,7 @@ EXPORTED = ["orthdion_create", "orthdion_destroy", "orthdion_set_dtypes", "orthd
             "orthdion_set_scale", "orthdion_set_ef", "orthdion_set_engine", "orthdion_set_passes",
             "orthdion_workspace_bytes", "orthdion_workspace_bytes_grouped", "orthdion_step",
             "orthdion_step_grouped", "orthdion_step_noalloc", "orthdion_get_factors", "orthdion_last_status",
-            "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_rank_policy",
+            "orthdion_set_concurrency", "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_rank_policy",
             "orthdion_resize_factor", "orthdion_version",
             "orthdion_launch_count", "orthdion_profile_begin", "orthdion_profile_end", "orthdion_stage_count",
             "orthdion_stage_name"]
@@ -228,6 +229,11 @@ def orthdion_step_grouped(table: PointerTable, workspace, stream=None):
                                        _dev_ptr(workspace, "workspace"),
                                        workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
            "orthdion_step_grouped")
+
+
+def orthdion_set_concurrency(lanes: int):
+    """Number of internal streams a grouped call spreads its launch batches over (1: none)."""
+    _check(lib().orthdion_set_concurrency(lanes), "orthdion_set_concurrency")
 
 
 def orthdion_get_factors(hs, index, workspace, shapes):

@@ -1,8 +1,9 @@
-// Host side of liborthdion: plans, workspace layout, sort-and-pack batching and the stage
-// sequence of one optimizer step.  All device work is enqueued on the caller's stream.
+// Host side of liborthdion: plans, workspace layout, packing of equal plans into launch batches
+// and the stage sequence of one optimizer step.  All device work is enqueued on the caller's stream.
 #include "../../include/orthdion.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -155,19 +156,63 @@ Layout make_layout(const orthdion_t* hs, int32_t count, size_t scratch_bytes) {
         }                                                                  \
     } while (0)
 
+// Kernel attributes (dynamic shared-memory limits) belong to a device: they are set once per
+// device ordinal, on the first step call made with that device current.
 int ensure_attributes() {
-    static int state = 0;   // 0 unknown, 1 ok, -1 failed
-    if (state) return state > 0 ? 0 : ORTHDION_ERR_CUDA;
+    static std::mutex mu;
+    static signed char state[kMaxDevices] = {};   // 0 unknown, 1 ok, -1 failed
+    int dev = -1;
+    CU_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return ORTHDION_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (state[dev]) return state[dev] > 0 ? 0 : ORTHDION_ERR_CUDA;
     cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)CH_SMEM_BYTES);
     if (e == cudaSuccess) e = tensor_engine_set_attributes();
     if (e != cudaSuccess) {
-        std::fprintf(stderr, "orthdion: kernel attribute setup failed: %s\n", cudaGetErrorString(e));
-        state = -1;
+        std::fprintf(stderr, "orthdion: kernel attribute setup failed on device %d: %s\n", dev, cudaGetErrorString(e));
+        state[dev] = -1;
         return ORTHDION_ERR_CUDA;
     }
-    state = 1;
+    state[dev] = 1;
     return 0;
+}
+
+// ---- internal streams of the grouped step ---------------------------------------------------
+// The steps of two launch batches (matrices of different plans) share nothing, so a grouped call
+// may run them side by side: the caller's stream forks into up to kMaxLanes internal streams,
+// every batch runs its whole stage sequence on one of them, and the caller's stream joins them
+// again before the call returns.  Order on the device is fixed by events only; the host never
+// waits.  The latency-bound r x r factor kernel of one batch and the ramp-up and tail of every
+// persistent kernel then overlap the kernels of the other batches.  Results per matrix do not
+// depend on this: every matrix goes through the same kernels with the same launch geometry.
+constexpr int kMaxLanes = 8;
+std::atomic<int> g_lanes{4};
+
+struct DeviceLanes {
+    std::mutex mu;                   // one grouped call at a time forks into the lanes of a device
+    bool ready = false;
+    cudaStream_t lane[kMaxLanes] = {};
+    cudaEvent_t fork = nullptr, done[kMaxLanes] = {};
+};
+
+// Lanes of the current device; streams and events are created on the first call that needs them
+// (no device memory is allocated).
+DeviceLanes* device_lanes() {
+    static DeviceLanes table[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    DeviceLanes* d = &table[dev];
+    std::lock_guard<std::mutex> lock(d->mu);
+    if (!d->ready) {
+        bool ok = cudaEventCreateWithFlags(&d->fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < kMaxLanes && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&d->lane[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&d->done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        d->ready = true;
+    }
+    return d;
 }
 
 template <class RA, class RB, class EP>
@@ -563,7 +608,31 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
         engine_error() = 0;
         const DiagBase db{reinterpret_cast<const int32_t*>(ws + lay.status_off),
                           reinterpret_cast<float*>(ws + lay.diag_off)};
-        run_group(cls, merged, db, st);
+        const int lanes = std::min<int>({g_lanes.load(), kMaxLanes, (int)cls.size()});
+        DeviceLanes* dl = lanes > 1 ? device_lanes() : nullptr;
+        if (dl) {
+            // heaviest batch first, each batch a lane of its own (round robin beyond `lanes`)
+            std::vector<int> order(cls.size());
+            for (size_t i = 0; i < cls.size(); ++i) order[i] = (int)i;
+            auto cost = [&](int i) {
+                const orthdion_plan* p = cls[i].p;
+                return (double)cls[i].b->count * ((double)p->m * p->n * p->r + (double)(p->m + p->n) * p->r * p->r);
+            };
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost(a) > cost(b); });
+            std::lock_guard<std::mutex> lock(dl->mu);
+            cudaEventRecord(dl->fork, st);
+            for (int l = 0; l < lanes; ++l) cudaStreamWaitEvent(dl->lane[l], dl->fork, 0);
+            for (size_t k = 0; k < order.size(); ++k) {
+                std::vector<ClassRun> one(1, cls[order[k]]);
+                run_group(one, merged, db, dl->lane[k % lanes]);
+            }
+            for (int l = 0; l < lanes; ++l) {
+                cudaEventRecord(dl->done[l], dl->lane[l]);
+                cudaStreamWaitEvent(st, dl->done[l], 0);
+            }
+        } else {
+            run_group(cls, merged, db, st);
+        }
         if (engine_error()) {
             std::fprintf(stderr, "orthdion: tensor map setup failed (%d)\n", engine_error());
             rc = ORTHDION_ERR_CUDA;
@@ -598,7 +667,6 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[ORTHDION_NOALLO
 namespace {
 // Device address of g_noalloc_scratch on the current device, looked up once per device.
 int noalloc_scratch_address(void** out) {
-    constexpr int kMaxDevices = 64;
     static std::mutex mu;
     static void* addr[kMaxDevices] = {};
     int dev = -1;
@@ -721,6 +789,12 @@ int orthdion_resize_factor(const float* Q_old, int64_t n, int32_t r_old, float* 
         std::fprintf(stderr, "orthdion: launch failed: %s\n", cudaGetErrorString(ce));
         return ORTHDION_ERR_CUDA;
     }
+    return ORTHDION_OK;
+}
+
+int orthdion_set_concurrency(int32_t lanes) {
+    if (lanes < 1 || lanes > kMaxLanes) return ORTHDION_ERR_INVALID_ARG;
+    g_lanes.store(lanes);
     return ORTHDION_OK;
 }
 

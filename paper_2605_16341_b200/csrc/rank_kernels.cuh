@@ -1,6 +1,6 @@
 // Resize of the warm-start factor for the adaptive-rank rule (appendix algorithm "Ada-Orth-Dion
-// Rank Selection": "resize U, V to rank r_{t+1} (truncate or pad)").  Only V (here Q, n x r) is
-// carried between steps; U (here P) is recomputed by every step.
+// Rank Selection", its last step: both factors are cut down or extended to the next rank).  Only
+// V (here Q, n x r) is carried between steps; U (here P) is recomputed by every step.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>

@@ -19,6 +19,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 
 #include "common.cuh"
@@ -1340,6 +1341,14 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
     }
 
     // ---------------- teardown ----------------
+    // A role that gave up on a bounded wait leaves bulk copies into this CTA's shared memory and
+    // issued MMAs possibly still in flight.  Nothing more is issued once the flag is up, so a fixed
+    // pause far longer than any copy or MMA takes (about a millisecond) lets them land before the
+    // shared memory and the tensor memory are given back.
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+    }
     tc_fence_before();
     __syncthreads();
     // pairs: neither CTA leaves (or frees tensor memory) while the other may still reach its barriers
@@ -1432,8 +1441,9 @@ inline TensorMapEncodeFn tensor_map_encoder() {
     }
     return fn;
 }
-// First error met while preparing launches of the current step call (0 = none).
-inline int& engine_error() { static int e = 0; return e; }
+// First error met while preparing launches of the current step call (0 = none); one per host
+// thread, so that concurrent step calls do not see each other's.
+inline int& engine_error() { static thread_local int e = 0; return e; }
 
 // 5-d map over the images `img` of all matrices of a batch: (64 bf16, rows, panels, terms, matrix),
 // with the box (64, box_rows, box_panels, box_terms, 1).  The images are stored pre-swizzled, so
@@ -1459,13 +1469,18 @@ inline void encode_img_map(CUtensorMap* map, const Batch& b, const ImgRef& img, 
     }
 }
 
+// Multiprocessor count of the current device (looked up once per device ordinal).
+constexpr int kMaxDevices = 64;
 inline int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
+    static std::atomic<int> cached[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= kMaxDevices) dev = 0;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n <= 0) {
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         if (n <= 0) n = 148;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
     return n;
 }

@@ -12,6 +12,13 @@ from paper_2605_16341_b200 import workloads as wl
 TOL_STEP = 1e-4       # ||dX_gpu - dX_or||_F / ||dX_or||_F after one step from identical state
 TOL_CHAIN = 1e-3      # the same after 10 chained steps
 TOL_ORTHO = 1e-5      # max |Q^T Q - I|
+# Largest element-wise error, relative to the largest element of the reference.  An error of
+# relative Frobenius size e spread evenly over N entries has its largest entry near
+# sqrt(2 ln N) ~ 6 times the error's root mean square, and the reference's largest entry is
+# about as many of its own root mean squares away, so a result inside TOL_STEP has a largest
+# error of about TOL_STEP of the largest reference entry (twice that is allowed); a localised fault (one wrong tile, one
+# dropped depth block) exceeds this while barely moving the Frobenius norm.
+TOL_MAXABS = 2e-4
 
 
 def poisoned_workspace(nbytes: int) -> torch.Tensor:
@@ -29,6 +36,31 @@ def f64(t: torch.Tensor) -> np.ndarray:
 
 def rel(a, b):
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def rel_max(a, b):
+    """Largest element-wise difference over the largest reference element."""
+    return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-300))
+
+
+def bf16_steps_apart(x_dev, x_ref32, x_before, slack):
+    """Distance between stored bf16 weights and reference values that are already rounded to bf16,
+    in units of the bf16 spacing at the magnitude of the weight (the larger of the old and the new
+    value, so that a weight that the update happens to cancel is not measured in the tiny steps
+    near zero), after taking off `slack`, the per-entry bound on the error of the single-pass
+    product that feeds the update.  Returns (largest distance, fraction of entries that differ)."""
+    a = x_dev.detach().float().cpu().numpy().astype(np.float64)
+    b = np.asarray(x_ref32, dtype=np.float64)
+    mag = np.maximum(np.abs(b), np.abs(x_before.detach().float().cpu().numpy().astype(np.float64)))
+    unit = np.maximum(mag, 2.0 ** -126) * 2.0 ** -8        # spacing is between 2^-8 and 2^-7 of the value
+    d = np.abs(a - b)
+    return float((np.maximum(d - slack, 0.0) / unit).max()), float(np.count_nonzero(d) / d.size)
+
+
+def single_pass_slack(P, Q, eta, scale=1.0, bits=8):
+    """Per-entry bound on the error of eta*scale*(P Q^T) when the product is one tensor-core pass
+    with operands rounded to `bits` significant bits: 2^-bits * sum_k |p_ik q_jk|."""
+    return eta * scale * (np.abs(f64(P)) @ np.abs(f64(Q)).T) * 2.0 ** -bits
 
 
 class GpuMatrix:

@@ -12,8 +12,8 @@ from oracle import orthdion_oracle as orc
 from paper_2605_16341_b200 import binding as od
 from paper_2605_16341_b200 import workloads as wl
 
-from parity_util import (TOL_CHAIN, TOL_ORTHO, TOL_STEP, GpuMatrix, check_bf16_rounding,
-                         delta_x_from_factors, f64, oracle_mode, poisoned_workspace, rel)
+from parity_util import (TOL_CHAIN, TOL_ORTHO, TOL_STEP, GpuMatrix, bf16_steps_apart, check_bf16_rounding,
+                         delta_x_from_factors, f64, oracle_mode, poisoned_workspace, rel, single_pass_slack)
 
 pytestmark = pytest.mark.gpu
 
@@ -209,7 +209,7 @@ def test_ill_conditioned_projection_takes_shifted_path(engine):
     P, _ = gm.factors()
     Pn = f64(P)
     assert np.isfinite(Pn).all()
-    assert np.abs(Pn.T @ Pn - np.eye(r)).max() <= 1e-4
+    assert np.abs(Pn.T @ Pn - np.eye(r)).max() <= TOL_ORTHO
     # the well-conditioned leading directions agree with the oracle
     ref = orc.step(f64(X), f64(M), f64(G), f64(Q), eta=0.01, mu=0.95)
     assert np.abs(Pn[:, :8] - ref["P"][:, :8]).max() <= 1e-3
@@ -270,36 +270,102 @@ def test_state_is_only_m_and_q(engine):
         x.close()
 
 
-# ------------------------------------------------------------------ cfg1: 4096 x 4096, r = 256, bf16
-@pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("fused", ["bf16x3", "fp16"])
-def test_cfg1_first_steps(mode, fused):
-    w = wl.workload("cfg1")
-    spec = w.matrices[0]
-    X, M, Q = wl.initial_state(spec, 0, 0)
-    basis = wl.grad_basis(w, spec, 0, 0)
-    gm = GpuMatrix(spec, X, M, Q, mu=w.mu, eta=w.eta, wd=w.wd, mode=mode,
-                   passes={2: 1, 3: 1} if fused == "fp16" else {2: 3, 3: 1})
-    Xo, Mo, Qo = f64(X), f64(M), f64(Q)
-    for t in range(3):
-        G = wl.gradient(w, spec, 0, 0, t, basis)
-        xb = gm.X.clone()
-        gm.step(G)
-        assert gm.status() == 0
-        ref = orc.step(Xo, Mo, f64(G), Qo, eta=w.eta, mu=w.mu, wd=w.wd, mode=oracle_mode(mode))
-        P, R = gm.factors()
-        dx_gpu = delta_x_from_factors(P, gm.Q, xb, w.eta, w.wd, 1.0)
-        dx_ref = ref["X"] - Xo
+# ------------------------------------------------------------------ chained steps with bf16 storage
+def chain_compare(w, specs, ids, steps, mode, passes=None, seed=0):
+    """`steps` chained steps of the matrices `ids` of workload `w`, as one grouped call per step.
+    The device carries its own state (bf16 X, fp32 M and Q); the oracle carries its own (float64
+    M and Q, and X rounded to bf16 after every step, which is what storing it means).  Per step
+    and matrix: dX formed in float64 from the device's fp32 factors against the oracle's, M, the
+    orthonormality of P and Q, the stored weights against the oracle's rounded ones."""
+    dev = torch.device("cuda")
+    hs, Xs, Ms, Qs, bases, state = [], [], [], [], [], []
+    for i in ids:
+        spec = specs[i]
+        h = od.orthdion_create(spec.m, spec.n, spec.r, w.mu, w.eta, w.wd, mode)
+        od.orthdion_set_dtypes(h, spec.x_dtype, spec.g_dtype)
+        for k, v in (passes or {}).items():
+            od.orthdion_set_passes(h, k, v)
+        hs.append(h)
+        X, M, Q = wl.initial_state(spec, seed, i)
+        bases.append(wl.grad_basis(w, spec, seed, i))
+        state.append([f64(X), f64(M), f64(Q)])
+        Xs.append(X.to(dev)); Ms.append(M.to(dev)); Qs.append(Q.to(dev))
+    ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
+    worst = dict(dx=0.0, M=0.0, ulps=0.0, differ=0.0)
+    for t in range(steps):
+        Gs = [wl.gradient(w, specs[i], seed, i, t, bases[k]) for k, i in enumerate(ids)]
+        Gd = [g.to(dev) for g in Gs]
+        Xb = [x.clone() for x in Xs]
+        od.orthdion_step_grouped(od.PointerTable(hs, Xs, Ms, Gd, Qs), ws)
+        torch.cuda.synchronize()
+        assert od.orthdion_last_status(hs, ws) == [0] * len(hs)
         tol = TOL_STEP if t == 0 else TOL_CHAIN
-        assert rel(dx_gpu, dx_ref) <= tol, (t, rel(dx_gpu, dx_ref))
-        assert rel(f64(gm.M), ref["M"]) <= tol
-        assert check_bf16_rounding(gm.X, xb, P, gm.Q, w.eta, w.wd, 1.0) <= 1.0 + 1e-6
-        Pn, Qn = f64(P), f64(gm.Q)
-        assert np.abs(Pn.T @ Pn - np.eye(spec.r)).max() <= TOL_ORTHO
-        if mode == od.MODE_ORTH:
-            assert np.abs(Qn.T @ Qn - np.eye(spec.r)).max() <= TOL_ORTHO
-        # the oracle carries the bf16-stored weights forward, like the device does
-        Xo, Mo, Qo = f64(gm.X), ref["M"], ref["Q"]
+        for k, i in enumerate(ids):
+            spec = specs[i]
+            Xo, Mo, Qo = state[k]
+            ref = orc.step(Xo, Mo, f64(Gs[k]), Qo, eta=w.eta, mu=w.mu, wd=w.wd, mode=oracle_mode(mode))
+            assert ref["status"] == orc.STATUS_OK
+            P, R = od.orthdion_get_factors(hs, k, ws, (spec.m, spec.n, spec.r))
+            dx_gpu = delta_x_from_factors(P, Qs[k], Xb[k], w.eta, w.wd, 1.0)
+            e_dx, e_m = rel(dx_gpu, ref["X"] - Xo), rel(f64(Ms[k]), ref["M"])
+            assert e_dx <= tol and e_m <= tol, (spec.name, t, e_dx, e_m)
+            Pn, Qn = f64(P), f64(Qs[k])
+            assert np.abs(Pn.T @ Pn - np.eye(spec.r)).max() <= TOL_ORTHO
+            if mode == od.MODE_ORTH:
+                assert np.abs(Qn.T @ Qn - np.eye(spec.r)).max() <= TOL_ORTHO
+            assert check_bf16_rounding(Xs[k], Xb[k], P, Qs[k], w.eta, w.wd, 1.0) <= 1.0 + 1e-6
+            # stored weights: the oracle's X', rounded to bf16 like the device's.  An entry whose
+            # exact value lies within the product's error of a rounding boundary may land on the
+            # other side of it, and keeps that one-step distance in later steps.
+            x_ref = orc.round_to_bf16(ref["X"])
+            ulps, differ = bf16_steps_apart(Xs[k], x_ref, Xb[k], single_pass_slack(P, Qs[k], w.eta))
+            assert ulps <= 2.0 and differ <= 0.02, (spec.name, t, ulps, differ)
+            state[k] = [x_ref.astype(np.float64), ref["M"], ref["Q"]]
+            worst = dict(dx=max(worst["dx"], e_dx), M=max(worst["M"], e_m), ulps=max(worst["ulps"], ulps),
+                         differ=max(worst["differ"], differ))
+    print(f"{w.name} mode {mode} passes {passes} {steps} chained steps: worst {worst}")
+    for h in hs:
+        od.orthdion_destroy(h)
+    return worst
+
+
+# cfg1: 4096 x 4096, r = 256, bf16 X and G.  Ten steps with the default passes (the fused pass as
+# one fp16 pass), three with the error-feedback product from split terms.
+@pytest.mark.parametrize("mode,fused,steps", [(od.MODE_ORTH, "default", 10), (od.MODE_COLNORM, "default", 10),
+                                              (od.MODE_ORTH, "bf16x3", 3), (od.MODE_COLNORM, "bf16x3", 3)])
+def test_cfg1_chained_steps(mode, fused, steps):
+    w = wl.workload("cfg1")
+    chain_compare(w, w.matrices, [0], steps, mode, passes=None if fused == "default" else {2: 3, 3: 1})
+
+
+# One matrix of every shape class of the 1.1B-shape model (2048 x 2048, 5632 x 2048, 2048 x 5632,
+# r = 512), stepped together for ten steps with the default passes.
+def test_cfg3_ten_chained_steps_of_one_matrix_per_shape_class():
+    w = wl.workload("cfg3", layers=1)
+    ids = [i for i, s in enumerate(w.matrices) if s.name in ("l0.q", "l0.gate", "l0.down")]
+    assert len(ids) == 3
+    chain_compare(w, w.matrices, ids, 10, od.MODE_ORTH)
+
+
+# The accuracy of the single-pass fused products before any storage rounding: fp32 weights (so
+# that X' itself can be compared) stepped with the passes a bf16 weight matrix gets by default.
+@pytest.mark.parametrize("mode", MODES)
+def test_single_pass_update_accuracy_on_fp32_weights(mode):
+    spec, X, M, G, Q = make_problem(1000, 1032, 256, F32, BF16, seed=77)
+    gm = GpuMatrix(spec, X, M, Q, mu=0.95, eta=0.01, mode=mode, passes={2: 1, 3: 1})
+    gm.step(G)
+    assert gm.status() == 0
+    ref = orc.step(f64(X), f64(M), f64(G), f64(Q), eta=0.01, mu=0.95, mode=oracle_mode(mode))
+    P, _ = gm.factors()
+    dx_applied = f64(gm.X) - f64(X)                       # what the fused pass really subtracted
+    dx_factors = delta_x_from_factors(P, gm.Q, X, 0.01, 0.0, 1.0)
+    dx_ref = ref["X"] - f64(X)
+    e_applied, e_factors = rel(dx_applied, dx_ref), rel(dx_factors, dx_ref)
+    print(f"single-pass update, mode {mode}: applied dX rel err {e_applied:.3e}, from fp32 factors {e_factors:.3e}")
+    # the factors meet the step tolerance; the applied update carries the rounding of one
+    # 11-bit-operand pass on top (2^-11 per operand: a few 1e-4), and the fp32 storage of X
+    assert e_factors <= TOL_STEP
+    assert e_applied <= 1e-3
     gm.close()
 
 
