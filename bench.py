@@ -33,6 +33,7 @@ sys.path.insert(0, ROOT)
 from paper_2605_16341_b200 import sharding  # noqa: E402
 from paper_2605_16341_b200 import workloads as wl  # noqa: E402
 
+DEFAULT_LANES = 4      # the library's default number of internal streams of a grouped call
 METRIC = "orthdion_step_param_elements_per_s"
 UNIT = "param-elements/s"
 
@@ -302,9 +303,6 @@ def run_ours(args):
     if sampler:
         sampler.start()
         time.sleep(0.3)
-    profile_on = not args.no_profile
-    if profile_on:
-        od.orthdion_profile_begin(max(1024, (launches_per_step + 16) * args.steps))
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(); torch.cuda.synchronize()
     l0 = od.orthdion_launch_count()
@@ -316,9 +314,28 @@ def run_ours(args):
     torch.cuda.synchronize(); barrier()
     t_wall1 = time.time()
     launches = od.orthdion_launch_count() - l0
-    stage_ms = od.orthdion_profile_end() if profile_on else {}
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     ms_total = sharding.max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
+
+    # Per-stage times: a second timed region of the same K steps with every launch bracketed by
+    # CUDA events on its stream.  It runs on ONE stream (lanes = 1): event pairs taken on the
+    # overlapping internal streams of the default configuration would not add up to the step.
+    profile_on = not args.no_profile
+    stage_ms, ms_step_one_stream = {}, None
+    if profile_on:
+        od.orthdion_set_concurrency(1)
+        step(args.warmup + args.steps)                       # settle into the one-stream order
+        torch.cuda.synchronize()
+        od.orthdion_profile_begin(max(1024, (launches_per_step + 16) * args.steps))
+        pv0, pv1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pv0.record(stream)
+        for k in range(args.steps):
+            step(args.warmup + args.steps + 1 + k)
+        pv1.record(stream)
+        torch.cuda.synchronize()
+        stage_ms = od.orthdion_profile_end()
+        ms_step_one_stream = pv0.elapsed_time(pv1) / args.steps
+        od.orthdion_set_concurrency(args.lanes or DEFAULT_LANES)
     ms_step = ms_total / args.steps
     flags = od.orthdion_last_status(hs, ws, stream)
     failed = sum(1 for f in flags if f & (od.STATUS_RANK_DEFICIENT | od.STATUS_NONFINITE | od.STATUS_WAIT_LIMIT))
@@ -414,6 +431,7 @@ def run_ours(args):
                                f"bf16 X/G, fp32 M, mode {args.mode}",
                    "engine": args.engine, "l2": "inputs (tens of GB per step) far exceed the 126 MB L2",
                    "grad_sets": args.grad_sets, "replicas": world, "diagnostics": args.diagnostics,
+                   "lanes": args.lanes or DEFAULT_LANES,
                    "diagnostics_summary": diag_summary,
                    "matrices_failed": failed, "matrices_shifted_qr": shifted},
         "clocks": clocks,
@@ -425,6 +443,9 @@ def run_ours(args):
                           "logical_tflop": (gemm_f + qr_f) / 1e12,
                           "peaks": peaks},
         "stages": stages,
+        "stages_region": ("second timed region of the same steps on one stream (lanes = 1), every launch between "
+                          "two CUDA events on its stream" if stage_ms else None),
+        "ms_per_step_one_stream": ms_step_one_stream,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)

@@ -86,8 +86,10 @@ typedef struct orthdion_plan* orthdion_t;
 
 /* Create a plan for m x n matrices at rank r (inputs of Algorithm 1: step size eta, EF
  * coefficient; mu gives the default (a, b) = (1, 1 - mu)).  Defaults: X and G bfloat16,
- * scale = 1, engine TENSOR.  The TENSOR engine needs r % 16 == 0, n % 8 == 0; SIMT any r.
- * Host memory only. */
+ * scale = 1, engine TENSOR.  The TENSOR engine needs r % 16 == 0, n % 8 == 0 and takes
+ * r <= 4096 (the rank fraction 0.25 of the paper's 16384-wide blocks); SIMT takes any
+ * r <= 1024 and is chosen when the TENSOR conditions do not hold.  Diagnostics need r <= 1024.
+ * ORTHDION_ERR_RANK otherwise.  Host memory only. */
 int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r,
                     float mu, float eta, float wd, int32_t mode);
 int orthdion_destroy(orthdion_t h);
@@ -133,6 +135,34 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count,
  * grouped call on a device creates that device's internal streams and events (no device memory);
  * two grouped calls on the same device are serialised on the host while they enqueue. */
 int orthdion_set_concurrency(int32_t lanes);
+
+/* Column-sharded step: one weight matrix split by columns over k ranks (the paper's FSDP setting,
+ * Section 2, "FSDP communication": only O((m + n) r) numbers cross the ranks per step).  Rank j
+ * holds X_j, M_j, G_j (m x n_j, its columns) and Q_j (n_j x r, the matching rows of the right
+ * factor); its plan is created with (m, n_j, r).  Since B Q_prev = sum_j B_j Q_j, R_j = B_j^T P and
+ * R^T R = sum_j R_j^T R_j, the step is a sequence of local phases with one sum over the ranks of a
+ * small fp32 buffer between two phases.  The caller makes that sum (an all-reduce on real ranks)
+ * in place on the buffer that orthdion_shard_reduce_buffer returns for the phase just run, then
+ * runs the next phase:
+ *   phase 0   Y_j = (M_j + G_j) Q_j                        reduce: Y, m x r
+ *   phase 1   P = orth(Y), the same on every rank; R_j = (M_j + G_j)^T P;
+ *             ORTH: Gram matrix of R_j                      reduce: r x r  (entries above the
+ *                                                           256 x 256 diagonal tiles are not used)
+ *             COLNORM: squared column norms of R_j          reduce: r
+ *   phase 2   ORTH: first CholeskyQR pass of R_j with the summed Gram matrix, Gram matrix of the
+ *             result                                        reduce: r x r
+ *             COLNORM: Q_j = R_j / norms; X_j, M_j updated: the step is complete
+ *   phase 3   ORTH only: second pass, Q_j; X_j, M_j updated: the step is complete
+ * Every phase is enqueued on `stream`; the same workspace (orthdion_workspace_bytes of the plan)
+ * must be passed to all phases of a step and keeps P, R_j and the status word afterwards
+ * (orthdion_get_factors, orthdion_last_status with count 1).  TENSOR engine only, diagnostics
+ * off.  The right QR is CholeskyQR2 here: a third pass that the second one asks for
+ * (ORTHDION_STATUS_SHIFTED_RIGHT) is reported but not taken.  With one shard and no reduction the
+ * phases compute what orthdion_step computes. */
+int orthdion_shard_phase(orthdion_t h, int32_t phase, void* X, float* M, const void* G, float* Q,
+                         void* workspace, size_t workspace_bytes, void* stream);
+/* Device pointer and length (in floats) of the buffer to sum over the ranks after `phase`. */
+int orthdion_shard_reduce_buffer(orthdion_t h, int32_t phase, void* workspace, float** buffer, int64_t* count);
 
 /* One step for one matrix without any caller-provided workspace and without any device-memory
  * allocation.  (The paper has no counterpart: this entry point exists for the integration, not

@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.orthdion_get_factors.argtypes = [pvp, i32, i32, vp, pvp, pvp]
     L.orthdion_last_status.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(i32)]
     L.orthdion_set_concurrency.argtypes = [i32]
+    L.orthdion_shard_phase.argtypes = [vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    L.orthdion_shard_reduce_buffer.argtypes = [vp, i32, vp, pvp, ctypes.POINTER(i64)]
     L.orthdion_set_diagnostics.argtypes = [vp, i32]
     L.orthdion_last_diagnostics.argtypes = [pvp, i32, vp, vp, ctypes.POINTER(ctypes.c_float)]
     dbl = ctypes.c_double
@@ -95,7 +97,7 @@ def lib() -> ctypes.CDLL:
     L.orthdion_stage_name.restype = ctypes.c_char_p
     for name in ("create", "destroy", "set_dtypes", "set_lr", "set_scale", "set_ef", "set_engine",
                  "set_passes", "step", "step_grouped", "step_noalloc", "get_factors", "last_status",
-                 "set_diagnostics", "last_diagnostics", "rank_policy", "resize_factor", "set_concurrency"):
+                 "set_diagnostics", "last_diagnostics", "rank_policy", "resize_factor", "set_concurrency", "shard_phase", "shard_reduce_buffer"):
         getattr(L, "orthdion_" + name).restype = i32
     _lib = L
     return L
@@ -105,7 +107,7 @@ EXPORTED = ["orthdion_create", "orthdion_destroy", "orthdion_set_dtypes", "orthd
             "orthdion_set_scale", "orthdion_set_ef", "orthdion_set_engine", "orthdion_set_passes",
             "orthdion_workspace_bytes", "orthdion_workspace_bytes_grouped", "orthdion_step",
             "orthdion_step_grouped", "orthdion_step_noalloc", "orthdion_get_factors", "orthdion_last_status",
-            "orthdion_set_concurrency", "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_rank_policy",
+            "orthdion_set_concurrency", "orthdion_shard_phase", "orthdion_shard_reduce_buffer", "orthdion_set_diagnostics", "orthdion_last_diagnostics", "orthdion_rank_policy",
             "orthdion_resize_factor", "orthdion_version",
             "orthdion_launch_count", "orthdion_profile_begin", "orthdion_profile_end", "orthdion_stage_count",
             "orthdion_stage_name"]
@@ -229,6 +231,23 @@ def orthdion_step_grouped(table: PointerTable, workspace, stream=None):
                                        _dev_ptr(workspace, "workspace"),
                                        workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
            "orthdion_step_grouped")
+
+
+def orthdion_shard_phase(h, phase, X, M, G, Q, workspace, stream=None):
+    """One local phase of the column-sharded step (X, M, G: this rank's columns; Q: its rows)."""
+    _check(lib().orthdion_shard_phase(h, phase, _dev_ptr(X, "X"), _dev_ptr(M, "M"), _dev_ptr(G, "G"), _dev_ptr(Q, "Q"),
+                                      _dev_ptr(workspace, "workspace"), workspace.numel() * workspace.element_size(),
+                                      _stream_ptr(stream)), "orthdion_shard_phase")
+
+
+def orthdion_shard_reduce_buffer(h, phase, workspace) -> torch.Tensor:
+    """The fp32 buffer inside `workspace` that has to be summed over the ranks after `phase`
+    (a flat torch view: all-reduce it in place)."""
+    buf, cnt = ctypes.c_void_p(), ctypes.c_int64()
+    _check(lib().orthdion_shard_reduce_buffer(h, phase, _dev_ptr(workspace, "workspace"), ctypes.byref(buf),
+                                              ctypes.byref(cnt)), "orthdion_shard_reduce_buffer")
+    off = (buf.value - workspace.data_ptr()) // 4
+    return workspace.view(torch.float32)[off:off + cnt.value]
 
 
 def orthdion_set_concurrency(lanes: int):

@@ -352,8 +352,11 @@ chol_inv_kernel(const __grid_constant__ Batch batch, CholArgs a) {
 
 // ---- ColNorm (Alg. 1, normalisation step, Dion branch): Q[:,j] = R[:,j] / ||R[:,j]||_2 ----------------------
 // One CTA per 32 columns: 32 x 32 threads, lanes along columns (coalesced rows).
+// part: 0 = the whole operation; 1 = only the squared column norms of the rows at hand, left at
+// cnorm_off (a column-sharded matrix sums them over the shards before it scales); 2 = only the
+// scaling, with the squared norms taken from cnorm_off.
 __global__ void __launch_bounds__(1024)
-colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t cnorm_off) {
+colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t cnorm_off, int part_sel) {
     const MatWork& w = batch.w[blockIdx.z];
     if (*w.status & ST_FAILED) return;
     __shared__ float part[32][33];
@@ -361,23 +364,61 @@ colnorm_kernel(const __grid_constant__ Batch batch, int64_t n, int r, int64_t cn
     const int lane = threadIdx.x % 32, ry = threadIdx.x / 32;
     const int j = blockIdx.x * 32 + lane;
     float s = 0.f;
-    if (j < r)
+    if (j < r && part_sel != 2)
         for (int64_t i = ry; i < n; i += 32) { float v = w.R[i * r + j]; s = fmaf(v, v, s); }
     part[ry][lane] = s;
     __syncthreads();
     if (ry == 0) {
         float t = 0.f;
-        for (int k = 0; k < 32; ++k) t += part[k][lane];
-        if (cnorm_off >= 0 && j < r) reinterpret_cast<float*>(w.scratch + cnorm_off)[j] = t;
+        if (part_sel == 2) {
+            if (j < r) t = reinterpret_cast<const float*>(w.scratch + cnorm_off)[j];
+        } else {
+            for (int k = 0; k < 32; ++k) t += part[k][lane];
+            if (cnorm_off >= 0 && j < r) reinterpret_cast<float*>(w.scratch + cnorm_off)[j] = t;
+        }
         float nrm = sqrtf(t);
-        if (j < r && !(nrm > 0.f)) atomicOr(w.status, ST_ZEROCOL);
+        if (j < r && !(nrm > 0.f) && part_sel != 1) atomicOr(w.status, ST_ZEROCOL);
         inv[lane] = (nrm > 0.f) ? 1.f / nrm : 0.f;
     }
     __syncthreads();
-    if (j < r) {
+    if (j < r && part_sel != 1) {
         const float sc = inv[lane];
         for (int64_t i = ry; i < n; i += 32) w.Q[i * r + j] = w.R[i * r + j] * sc;
     }
+}
+
+// ---- helpers of the column-sharded step ---------------------------------------------------------
+// Column sums of squares of an fp32 matrix S (rows x r) per block of 32 rows, in the layout the
+// product kernels write next to their results: out[blk * r + j], blk < 4 * ceil(rows / 128)
+// (blocks beyond the matrix hold zeros).  One CTA per (32-row block, 256 columns).
+__global__ void __launch_bounds__(256)
+colsq_blocks_kernel(const __grid_constant__ Batch batch, Sel src, int64_t rows, int r, int64_t colsq_off) {
+    const MatWork& w = batch.w[blockIdx.z];
+    if (*w.status & ST_FAILED) return;
+    const float* S = pick(w, src);
+    float* out = reinterpret_cast<float*>(w.scratch + colsq_off);
+    const int j = blockIdx.y * 256 + threadIdx.x;
+    if (j >= r) return;
+    const int64_t i0 = (int64_t)blockIdx.x * 32;
+    float s = 0.f;
+    for (int k = 0; k < 32; ++k)
+        if (i0 + k < rows) { const float v = S[(i0 + k) * r + j]; s = fmaf(v, v, s); }
+    out[(int64_t)blockIdx.x * r + j] = s;
+}
+
+// Gram diagonal <- sum of the per-block column sums of squares (fp32 sums: the tensor core's
+// truncating accumulation would bias the diagonal low), so that a reduction of the r x r matrix
+// over the shards carries the exact diagonal along.
+__global__ void __launch_bounds__(256)
+gram_diag_kernel(const __grid_constant__ Batch batch, Sel gram, int r, int64_t colsq_off, int blocks) {
+    const MatWork& w = batch.w[blockIdx.z];
+    if (*w.status & ST_FAILED) return;
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= r) return;
+    const float* cs = reinterpret_cast<const float*>(w.scratch + colsq_off);
+    float d = 0.f;
+    for (int b = 0; b < blocks; ++b) d += cs[(int64_t)b * r + j];
+    pick(w, gram)[(int64_t)j * r + j] = d;
 }
 
 __global__ void init_status_kernel(const __grid_constant__ Batch batch) {

@@ -19,6 +19,17 @@
 //   inv [[A, 0], [B, C]] = [[Ai, 0], [-Ci B Ai, Ci]]                   (tile products)
 // The later passes of a CholeskyQR see a Gram matrix I + E with E tiny; when a rigorous bound on
 // |E|_2 is small enough, L^{-1} = I - Phi(E) (first order) replaces the factorisation.
+//
+// MULTI form: one matrix per thread-block CLUSTER.  When a launch has fewer matrices than the
+// device has room for CTAs, a lone CTA per matrix leaves most of the device idle while it walks
+// its lists of tile products one after the other.  The CTAs of a cluster share one matrix: every
+// list of independent tile products (panel, trailing update, the two steps of the pairwise
+// inverse) and every copy loop is dealt out over the CTAs, the 32 x 32 diagonal blocks are
+// factored by CTA 0 alone, and phases are separated by cluster barriers.  The matrix stays in
+// global memory (L2); loads of data another CTA of the cluster may have written bypass L1
+// (ld.global.cg) and follow a release/acquire cluster barrier.  Decisions that steer control
+// flow (first-order inverse or not, breakdown, retry) are taken by CTA 0 and read by the others
+// from its shared memory, so all CTAs of a cluster always take the same path.
 #pragma once
 #include "common.cuh"
 #include "factor_kernels.cuh"
@@ -42,6 +53,29 @@ struct TcTask {
     float alpha, beta;
 };
 
+// ---- cluster helpers of the MULTI form ----------------------------------------------------
+__device__ __forceinline__ void ct_cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the int at `p` (a shared-memory variable of this kernel) as CTA 0 of the cluster holds it
+__device__ __forceinline__ int ct_read_cta0(const int* p) {
+    const uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(p));
+    uint32_t remote;
+    int v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(0));
+    asm volatile("ld.shared::cluster.b32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+    return v;
+}
+// loads of matrix data that another CTA of the cluster may have written: L2 only
+template <bool MULTI> __device__ __forceinline__ float ct_ld(const float* p) { return MULTI ? __ldcg(p) : *p; }
+template <bool MULTI> __device__ __forceinline__ float2 ct_ld2(const float* p) {
+    return MULTI ? __ldcg(reinterpret_cast<const float2*>(p)) : *reinterpret_cast<const float2*>(p);
+}
+template <bool MULTI> __device__ __forceinline__ float4 ct_ld4(const float* p) {
+    return MULTI ? __ldcg(reinterpret_cast<const float4*>(p)) : *reinterpret_cast<const float4*>(p);
+}
+
 __device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -50,8 +84,10 @@ __device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], const uint32_t (
 }
 
 // All 256 threads.  Warp w owns rows 16*(w % 4).., columns 32*(w / 4).. of the tile.
-__device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* stage) {
-    if (ntasks <= 0) return;
+// MULTI: this CTA takes the tasks first, first + stride, ... of the list (its share of a cluster's work).
+template <bool MULTI>
+__device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* stage, int first = 0, int stride = 1) {
+    if (ntasks <= first) return;
     __nv_bfloat16* Ah = stage;
     __nv_bfloat16* Al = Ah + 64 * CT_LDK;
     __nv_bfloat16* Bh = Al + 64 * CT_LDK;
@@ -72,13 +108,12 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
         const bool ak = k0 + a_kk < t.kend;
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-            ra[e] = (ak && a_ii + 16 * e < t.Mt) ? *reinterpret_cast<const float2*>(Ap + e * 16 * t.a_rs) : make_float2(0.f, 0.f);
+            ra[e] = (ak && a_ii + 16 * e < t.Mt) ? ct_ld2<MULTI>(Ap + e * 16 * t.a_rs) : make_float2(0.f, 0.f);
         if (t.b_rs == 1) {
             const float* Bp = t.B + (k0 + a_kk + a_ii * t.b_cs);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float2 v = (ak && a_ii + 16 * e < t.Nt) ? *reinterpret_cast<const float2*>(Bp + e * 16 * t.b_cs)
-                                                              : make_float2(0.f, 0.f);
+                const float2 v = (ak && a_ii + 16 * e < t.Nt) ? ct_ld2<MULTI>(Bp + e * 16 * t.b_cs) : make_float2(0.f, 0.f);
                 rb[2 * e] = v.x; rb[2 * e + 1] = v.y;
             }
         } else {
@@ -86,10 +121,10 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
             const float* Bp = t.B + ((k0 + kk) * t.b_rs + jj);
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-                rb[e] = (jj < t.Nt && k0 + kk + 4 * e < t.kend) ? Bp[e * 4 * t.b_rs] : 0.f;
+                rb[e] = (jj < t.Nt && k0 + kk + 4 * e < t.kend) ? ct_ld<MULTI>(Bp + e * 4 * t.b_rs) : 0.f;
         }
     };
-    int ti = 0, k0 = tasks[0].kbeg;
+    int ti = first, k0 = tasks[first].kbeg;
     load(ti, k0);
     float acc[4][4] = {};
     while (true) {
@@ -122,7 +157,7 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
         __syncthreads();
         const bool last_chunk = k0 + CT_KC >= tasks[ti].kend;
         int nti = ti, nk0 = k0 + CT_KC;
-        if (last_chunk) { nti = ti + 1; nk0 = nti < ntasks ? tasks[nti].kbeg : 0; }
+        if (last_chunk) { nti = ti + stride; nk0 = nti < ntasks ? tasks[nti].kbeg : 0; }
         const bool has_next = nti < ntasks;
         if (has_next) load(nti, nk0);
 #pragma unroll
@@ -160,8 +195,7 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
                         const int i = row0 + gq + h * 8, j = col0 + nf * 8 + tq * 2;
                         v0[nf][h] = i < t.Mt && j < t.Nt && !(t.lower_only && (t.cg0 + j > t.rg0 + i));
                         v1[nf][h] = i < t.Mt && j + 1 < t.Nt && !(t.lower_only && (t.cg0 + j + 1 > t.rg0 + i));
-                        cv2[nf][h] = (v0[nf][h] && t.beta != 0.f) ? *reinterpret_cast<const float2*>(t.C + i * t.c_rs + j)
-                                                                  : make_float2(0.f, 0.f);
+                        cv2[nf][h] = (v0[nf][h] && t.beta != 0.f) ? ct_ld2<MULTI>(t.C + i * t.c_rs + j) : make_float2(0.f, 0.f);
                     }
 #pragma unroll
                 for (int nf = 0; nf < 4; ++nf)
@@ -183,7 +217,7 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
                 for (int e = 0; e < 4; ++e) {
                     const int i = row0 + gq + (e / 2) * 8, j = col0 + nf * 8 + tq * 2 + (e % 2);
                     valid[nf][e] = i < t.Mt && j < t.Nt && !(t.lower_only && (t.cg0 + j > t.rg0 + i));
-                    cv[nf][e] = (valid[nf][e] && t.beta != 0.f) ? t.C[i * t.c_rs + j * t.c_cs] : 0.f;
+                    cv[nf][e] = (valid[nf][e] && t.beta != 0.f) ? ct_ld<MULTI>(t.C + i * t.c_rs + j * t.c_cs) : 0.f;
                 }
 #pragma unroll
             for (int nf = 0; nf < 4; ++nf)
@@ -201,25 +235,33 @@ __device__ void tc_run_tasks(const TcTask* tasks, int ntasks, __nv_bfloat16* sta
     __syncthreads();
 }
 
+template <bool MULTI>
 __global__ void __launch_bounds__(CT_THREADS, 2)
-chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
+chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a, int csize) {
     __shared__ __align__(16) __nv_bfloat16 s_stage[4 * 64 * CT_LDK];
     __shared__ TcTask s_tasks[CT_MAX_TASKS];
     __shared__ float s_blk[32 * 33];
     __shared__ float s_piv[32];
-    __shared__ float s_diag[1024];
-    __shared__ float s_rowsum[1024];
+    extern __shared__ float s_dyn[];          // 2 r floats: Gram diagonal, row sums of |Gram - I|
+    float* s_diag = s_dyn;
+    float* s_rowsum = s_dyn + a.r;
     __shared__ float red[8];
-    __shared__ int s_ntasks, s_fail, s_status;
+    __shared__ int s_ntasks, s_fail, s_status, s_decision;
     __shared__ float s_trace, s_dmin, s_dmax;
 
-    const MatWork& w = batch.w[blockIdx.x];
+    // MULTI: the csize CTAs of a cluster (ranks 0 .. csize-1) share matrix blockIdx.x / csize
+    const int crank = MULTI ? (int)(blockIdx.x % (unsigned)csize) : 0;
+    const int nshare = MULTI ? csize : 1;
+    const MatWork& w = batch.w[MULTI ? blockIdx.x / (unsigned)csize : blockIdx.x];
     const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
     const int r = a.r;
     const int shift_bit = a.which ? ST_SHIFT_R : ST_SHIFT_L;
+    auto phase_sync = [&]() { if (MULTI) ct_cluster_sync(); else __syncthreads(); };
 
     if (tid == 0) s_status = *w.status;
     __syncthreads();
+    // every CTA of the cluster has read the status word before any of them may change it
+    if (MULTI) ct_cluster_sync();
     const int st0 = s_status;
     if (st0 & ST_FAILED) return;
     if (a.pass == 3 && !(st0 & shift_bit)) return;
@@ -240,7 +282,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
                 d = A[i * r + i];
             }
             s_diag[i] = d;
-            if (a.cnorm_off >= 0) reinterpret_cast<float*>(w.scratch + a.cnorm_off)[i] = d;
+            if (a.cnorm_off >= 0 && crank == 0) reinterpret_cast<float*>(w.scratch + a.cnorm_off)[i] = d;
             t += d;
         }
         for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -254,8 +296,9 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         __syncthreads();
     }
     const float trace = s_trace;
+    // (the same sum in the same order in every CTA of a cluster: all of them take this exit or none)
     if (!(fabsf(trace) <= 3.0e38f)) {   // Inf or NaN
-        if (tid == 0) atomicOr(w.status, ST_NONFINITE);
+        if (tid == 0 && crank == 0) atomicOr(w.status, ST_NONFINITE);
         return;
     }
 
@@ -265,27 +308,30 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     // below CT_SERIES_LIMIT the dropped terms are below 2e-6 and the factorisation is skipped.
     bool series = false;
     if (a.pass >= 2) {
-        float colacc[32];
-#pragma unroll
-        for (int t = 0; t < 32; ++t) colacc[t] = 0.f;
         for (int i = tid; i < r; i += CT_THREADS) s_rowsum[i] = fabsf(s_diag[i] - 1.f);
         __syncthreads();
-        for (int i = warp; i < r; i += CT_THREADS / 32) {
-            float rs = 0.f;
+        // strictly lower entries, in column blocks of 1024 (32 column sums per lane in registers)
+        for (int cb = 0; cb < r; cb += 1024) {
+            float colacc[32];
 #pragma unroll
-            for (int t = 0; t < 32; ++t) {
-                const int j = lane + 32 * t;
-                if (j < i) {
-                    const float v = fabsf(A[i * r + j]);
-                    rs += v; colacc[t] += v;
+            for (int t = 0; t < 32; ++t) colacc[t] = 0.f;
+            for (int i = cb + warp; i < r; i += CT_THREADS / 32) {
+                float rs = 0.f;
+#pragma unroll
+                for (int t = 0; t < 32; ++t) {
+                    const int j = cb + lane + 32 * t;
+                    if (j < i) {
+                        const float v = fabsf(A[(size_t)i * r + j]);
+                        rs += v; colacc[t] += v;
+                    }
                 }
+                for (int o = 16; o; o >>= 1) rs += __shfl_xor_sync(0xffffffffu, rs, o);
+                if (lane == 0) atomicAdd(&s_rowsum[i], rs);
             }
-            for (int o = 16; o; o >>= 1) rs += __shfl_xor_sync(0xffffffffu, rs, o);
-            if (lane == 0) atomicAdd(&s_rowsum[i], rs);
-        }
 #pragma unroll
-        for (int t = 0; t < 32; ++t)
-            if (lane + 32 * t < r && colacc[t] != 0.f) atomicAdd(&s_rowsum[lane + 32 * t], colacc[t]);
+            for (int t = 0; t < 32; ++t)
+                if (cb + lane + 32 * t < r && colacc[t] != 0.f) atomicAdd(&s_rowsum[cb + lane + 32 * t], colacc[t]);
+        }
         __syncthreads();
         float mx = 0.f;
         for (int i = tid; i < r; i += CT_THREADS) mx = fmaxf(mx, s_rowsum[i]);
@@ -295,14 +341,22 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         mx = 0.f;
         for (int i = 0; i < CT_THREADS / 32; ++i) mx = fmaxf(mx, red[i]);
         series = mx <= CT_SERIES_LIMIT;          // false for NaN
+        if (MULTI) {
+            // the row sums are accumulated with shared-memory atomics, whose order may differ from
+            // CTA to CTA: CTA 0 decides for the cluster
+            if (tid == 0) s_decision = series ? 1 : 0;
+            ct_cluster_sync();
+            series = ct_read_cta0(&s_decision) != 0;
+            ct_cluster_sync();                   // nobody overwrites s_decision before all have read it
+        }
         // Second pass with Q1 far from orthonormal (cond(Y)^2 u was not small): its result will
         // not be orthonormal to working accuracy either, so ask for the third pass.
-        if (a.pass == 2 && !(mx <= CT_THIRD_PASS_LIMIT) && tid == 0) atomicOr(w.status, shift_bit);
+        if (a.pass == 2 && !(mx <= CT_THIRD_PASS_LIMIT) && tid == 0 && crank == 0) atomicOr(w.status, shift_bit);
         __syncthreads();
     }
     if (series) {
         const int r4 = r / 4;
-        for (int q = tid; q < r * r4; q += CT_THREADS) {
+        for (int q = tid + crank * CT_THREADS; q < r * r4; q += CT_THREADS * nshare) {
             const int i = q / r4, j4 = (q - i * r4) * 4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
             if (j4 <= i) {
@@ -315,16 +369,35 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
             }
             *reinterpret_cast<float4*>(W + i * r + j4) = v;
         }
-        __syncthreads();
+        phase_sync();
     }
 
+    // Task lists longer than the table are run in windows of CT_MAX_TASKS: thread 0 walks the whole
+    // list for every window and keeps the tasks that fall into it.
+    int gen_base = 0, gen_count = 0;
     auto add_task = [&](float* C, int c_rs, int c_cs, const float* A_, int a_rs, const float* B_, int b_rs, int b_cs,
                         int Mt, int Nt, int kbeg, int kend, float alpha, float beta, bool lower_only, int rg0, int cg0) {
-        TcTask& t = s_tasks[s_ntasks++];
+        const int k = gen_count++;
+        if (k < gen_base || k >= gen_base + CT_MAX_TASKS) return;
+        TcTask& t = s_tasks[k - gen_base];
         t.C = C; t.A = A_; t.B = B_;
         t.c_rs = c_rs; t.c_cs = c_cs; t.a_rs = a_rs; t.b_rs = b_rs; t.b_cs = b_cs;
         t.Mt = Mt; t.Nt = Nt; t.kbeg = kbeg; t.kend = kend; t.lower_only = lower_only ? 1 : 0; t.rg0 = rg0; t.cg0 = cg0;
         t.alpha = alpha; t.beta = beta;
+    };
+    // Runs the list of independent tile products that build() enumerates (always in the same
+    // order); MULTI: task k of the list goes to CTA k % nshare, and the cluster meets afterwards.
+    auto run_list = [&](auto build) {
+        for (int base = 0;; base += CT_MAX_TASKS) {
+            if (tid == 0) { gen_base = base; gen_count = 0; build(); s_ntasks = gen_count; }
+            __syncthreads();
+            const int total = s_ntasks;
+            const int first = MULTI ? ((crank - base % nshare) % nshare + nshare) % nshare : 0;
+            tc_run_tasks<MULTI>(s_tasks, min(CT_MAX_TASKS, total - base), s_stage, first, nshare);
+            __syncthreads();
+            if (base + CT_MAX_TASKS >= total) break;
+        }
+        if (MULTI) ct_cluster_sync();
     };
 
     bool ok = series;
@@ -335,7 +408,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
         // (eight loads in flight per thread: one at a time, the L2 round trips of this copy alone
         // were 8 % of the kernel)
         const int r4 = r / 4;
-        for (int q0 = tid; q0 < r * r4; q0 += 8 * CT_THREADS) {
+        for (int q0 = tid + crank * 8 * CT_THREADS; q0 < r * r4; q0 += 8 * CT_THREADS * nshare) {
             float4 v[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -359,7 +432,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
             }
         }
         if (tid == 0) { s_fail = 0; s_dmin = 3.0e38f; s_dmax = 0.f; }
-        __syncthreads();
+        phase_sync();
 
         for (int k0 = 0; k0 < r; k0 += CT_NB) {
             const int nb = min(CT_NB, r - k0);
@@ -367,11 +440,11 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
             // rank-one update by everybody, two barriers per column), then inverted by one warp
             // (thread c solves L x = e_c with x in registers; L(i, p) are broadcast reads).  The
             // inverse replaces the block in place right away: it is needed at the end anyway.
-            {
+            if (crank == 0) {
                 for (int e = tid; e < 1024; e += CT_THREADS) {
                     const int i = e >> 5, c = e & 31;
                     float v = (i == c) ? 1.f : 0.f;          // rows beyond nb are identity rows
-                    if (i < nb && c <= i) v = W[(k0 + i) * r + k0 + c];
+                    if (i < nb && c <= i) v = ct_ld<MULTI>(W + (k0 + i) * r + k0 + c);
                     s_blk[i * 33 + c] = v;
                 }
                 __syncthreads();
@@ -412,44 +485,46 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
                     }
                 }
             }
-            __syncthreads();
+            phase_sync();
             const int t0 = k0 + nb, s = r - t0;
             if (s > 0) {
                 // panel: rows below <- rows below * inv(L_kk)^T
-                if (tid == 0) {
-                    s_ntasks = 0;
+                run_list([&]() {
                     for (int i0 = 0; i0 < s; i0 += 64)
-                        add_task(W + (t0 + i0) * r + k0, r, 1, W + (t0 + i0) * r + k0, r, W + k0 * r + k0, 1, r,
-                                 min(64, s - i0), nb, 0, nb, 1.f, 0.f, false, 0, 0);
-                }
-                __syncthreads();
-                tc_run_tasks(s_tasks, s_ntasks, s_stage);
+                        add_task(W + (size_t)(t0 + i0) * r + k0, r, 1, W + (size_t)(t0 + i0) * r + k0, r,
+                                 W + (size_t)k0 * r + k0, 1, r, min(64, s - i0), nb, 0, nb, 1.f, 0.f, false, 0, 0);
+                });
                 // trailing update: W[t0+i][t0+j] -= sum_c W[t0+i][k0+c] W[t0+j][k0+c], j <= i
-                if (tid == 0) {
-                    s_ntasks = 0;
+                run_list([&]() {
                     const int nt = (s + 63) / 64;
                     for (int ti = 0; ti < nt; ++ti)
                         for (int tj = 0; tj <= ti; ++tj) {
                             const int ri = t0 + ti * 64, cj = t0 + tj * 64;
-                            add_task(W + ri * r + cj, r, 1, W + ri * r + k0, r, W + cj * r + k0, 1, r,
+                            add_task(W + (size_t)ri * r + cj, r, 1, W + (size_t)ri * r + k0, r, W + (size_t)cj * r + k0, 1, r,
                                      min(64, r - ri), min(64, r - cj), 0, nb, -1.f, 1.f, ti == tj, ri, cj);
                         }
-                }
-                __syncthreads();
-                tc_run_tasks(s_tasks, s_ntasks, s_stage);
+                });
             }
         }
-        const bool fail = s_fail != 0;
-        const bool ill = (a.pass == 1) && (s_dmax > a.cond_limit * s_dmin);
+        bool fail = s_fail != 0;
+        bool ill = (a.pass == 1) && (s_dmax > a.cond_limit * s_dmin);
+        if (MULTI) {
+            // only CTA 0 has factored the diagonal blocks: its verdict holds for the cluster
+            if (tid == 0) s_decision = (fail ? 1 : 0) | (ill ? 2 : 0);
+            ct_cluster_sync();
+            const int d = ct_read_cta0(&s_decision);
+            fail = (d & 1) != 0; ill = (d & 2) != 0;
+            ct_cluster_sync();
+        }
         if (!fail && !(ill && attempt == 0)) {
             ok = true;
         } else if (attempt == 0 && a.pass == 1) {
-            if (tid == 0) atomicOr(w.status, shift_bit);
+            if (tid == 0 && crank == 0) atomicOr(w.status, shift_bit);
         }
         __syncthreads();
     }
     if (!ok) {
-        if (tid == 0) atomicOr(w.status, ST_RANKDEF);
+        if (tid == 0 && crank == 0) atomicOr(w.status, ST_RANKDEF);
         return;
     }
 
@@ -457,47 +532,41 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     for (int s = CT_NB; s < r && !series; s *= 2) {
         const int npairs = (r + 2 * s - 1) / (2 * s);
         // step 1: T = B * Ai, kept transposed in the (unused, zero) mirror block above the diagonal
-        if (tid == 0) {
-            s_ntasks = 0;
+        run_list([&]() {
             for (int pr = 0; pr < npairs; ++pr) {
                 const int p = pr * 2 * s, sc = min(s, r - p - s);
                 if (sc <= 0) continue;
                 for (int i0 = 0; i0 < sc; i0 += 64)
                     for (int c0 = 0; c0 < s; c0 += 64)
-                        add_task(W + (p + c0) * r + (p + s + i0), 1, r,           // T(i,k) at W[p+k][p+s+i]
-                                 W + (p + s + i0) * r + p, r,                     // B(i,q)
-                                 W + p * r + (p + c0), r, 1,                      // Ai(q,k)
+                        add_task(W + (size_t)(p + c0) * r + (p + s + i0), 1, r,   // T(i,k) at W[p+k][p+s+i]
+                                 W + (size_t)(p + s + i0) * r + p, r,             // B(i,q)
+                                 W + (size_t)p * r + (p + c0), r, 1,              // Ai(q,k)
                                  min(64, sc - i0), min(64, s - c0), c0, s, 1.f, 0.f, false, 0, 0);
             }
-        }
-        __syncthreads();
-        tc_run_tasks(s_tasks, s_ntasks, s_stage);
+        });
         // step 2: B <- -Ci * T
-        if (tid == 0) {
-            s_ntasks = 0;
+        run_list([&]() {
             for (int pr = 0; pr < npairs; ++pr) {
                 const int p = pr * 2 * s, sc = min(s, r - p - s);
                 if (sc <= 0) continue;
                 for (int i0 = 0; i0 < sc; i0 += 64)
                     for (int c0 = 0; c0 < s; c0 += 64)
-                        add_task(W + (p + s + i0) * r + (p + c0), r, 1,           // Bnew(i,k)
-                                 W + (p + s + i0) * r + (p + s), r,               // Ci(i,q)
-                                 W + (p + c0) * r + (p + s), 1, r,                // T(q,k) at W[p+k][p+s+q]
+                        add_task(W + (size_t)(p + s + i0) * r + (p + c0), r, 1,   // Bnew(i,k)
+                                 W + (size_t)(p + s + i0) * r + (p + s), r,       // Ci(i,q)
+                                 W + (size_t)(p + c0) * r + (p + s), 1, r,        // T(q,k) at W[p+k][p+s+q]
                                  min(64, sc - i0), min(64, s - c0), 0, min(sc, i0 + 64), -1.f, 0.f, false, 0, 0);
             }
-        }
-        __syncthreads();
-        tc_run_tasks(s_tasks, s_ntasks, s_stage);
+        });
         // clear the mirror blocks again
         for (int pr = 0; pr < npairs; ++pr) {
             const int p = pr * 2 * s, sc = min(s, r - p - s);
             if (sc <= 0) continue;
-            for (int e = tid; e < s * sc; e += CT_THREADS) {
+            for (int e = tid + crank * CT_THREADS; e < s * sc; e += CT_THREADS * nshare) {
                 const int k = e / sc, i = e - k * sc;
                 W[(p + k) * r + (p + s + i)] = 0.f;
             }
         }
-        __syncthreads();
+        phase_sync();
     }
 
     // ---- split image of (L^{-1})^T for the tensor-core apply product ---------------------------
@@ -505,9 +574,9 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
     // operand MN-major (depth along image rows) in 256-column instructions.
     if (a.img.off >= 0) {
         unsigned char* __restrict__ scr = reinterpret_cast<unsigned char*>(w.scratch);
-        const float* __restrict__ Wr = W;
+        const float* Wr = W;
         const int chunks = a.img.panels * a.img.rows_pad * 8;
-        for (int q0 = tid; q0 < chunks; q0 += 4 * CT_THREADS) {
+        for (int q0 = tid + crank * 4 * CT_THREADS; q0 < chunks; q0 += 4 * CT_THREADS * nshare) {
             // consecutive threads take consecutive image rows (consecutive k: contiguous in W);
             // four chunks (32 loads) in flight per thread
             float v[4][8];
@@ -518,7 +587,7 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a) {
                 const int col = panel * 64 + c * 8;
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                    v[u][i] = (q < chunks && row < r && col + i < r) ? Wr[(col + i) * r + row] : 0.f;
+                    v[u][i] = (q < chunks && row < r && col + i < r) ? ct_ld<MULTI>(Wr + (col + i) * r + row) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {

@@ -35,7 +35,8 @@ struct orthdion_plan {
 namespace {
 
 constexpr uint32_t kMagic = 0x0D10A5E7u;
-constexpr int32_t kMaxRank = 1024;
+constexpr int32_t kMaxRank = 4096;        // tensor engine; the SIMT engine and the diagnostics take r <= 1024
+constexpr int32_t kMaxRankSimt = 1024;
 constexpr size_t kScratchBudget = (size_t)24 << 30;   // per launch batch
 constexpr float kShiftRel = 1e-5f;
 // max/min diag(L) of the first Cholesky above which the QR takes the shifted three-pass path.
@@ -168,6 +169,11 @@ int ensure_attributes() {
     if (state[dev]) return state[dev] > 0 ? 0 : ORTHDION_ERR_CUDA;
     cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)CH_SMEM_BYTES);
+    // the r x r factor kernel keeps 2 r floats in dynamic shared memory next to its static tables
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(chol_inv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kMaxRank * 4);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(chol_inv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kMaxRank * 4);
     if (e == cudaSuccess) e = tensor_engine_set_attributes();
     if (e != cudaSuccess) {
         std::fprintf(stderr, "orthdion: kernel attribute setup failed on device %d: %s\n", dev, cudaGetErrorString(e));
@@ -234,8 +240,10 @@ struct ClassRun {
 };
 
 // Cholesky + inverse of every class's Gram matrix: classes of equal (r, engine) share launches.
+// diag_from_gram: take the diagonal from the Gram matrix itself instead of the column-square
+// partials of the producing kernel (column-sharded matrices: the reduced Gram matrix carries it).
 void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int which, int pass,
-                Batch* merged, cudaStream_t st) {
+                Batch* merged, int call_matrices, cudaStream_t st, bool diag_from_gram = false) {
     std::vector<char> done(which_cls.size(), 0);
     for (size_t i = 0; i < which_cls.size(); ++i) {
         if (done[i]) continue;
@@ -247,15 +255,40 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
         ca.cond_limit = lead.tensor() ? kCondLimitTensor : kCondLimit;
         ca.colsq = sel(W_SCRATCH, 0); ca.use_colsq = 0; ca.img = no_img(); ca.cnorm_off = -1;
         if (lead.tensor()) {
-            ca.colsq = sel(W_SCRATCH, lead.sc.ts.colsq); ca.use_colsq = 1; ca.img = lead.sc.ts.linv;
+            ca.colsq = sel(W_SCRATCH, lead.sc.ts.colsq); ca.use_colsq = diag_from_gram ? 0 : 1; ca.img = lead.sc.ts.linv;
             if (which == 1 && pass == 1) ca.cnorm_off = lead.sc.ts.cnorm;
         }
         merged->count = 0; merged->pad = 0; merged->scratch_stride = 0;
         auto flush = [&]() {
             if (!merged->count) return;
             prof::Scope scope(prof::S_CHOL, st);
-            if (lead.tensor()) chol_inv_tc_kernel<<<merged->count, CT_THREADS, 0, st>>>(*merged, ca);
-            else chol_inv_kernel<<<merged->count, CH_THREADS, CH_SMEM_BYTES, st>>>(*merged, ca);
+            if (lead.tensor()) {
+                // Fewer matrices than the device has room for CTAs (two per multiprocessor): share
+                // each matrix among the CTAs of a cluster (2, 4 or 8).
+                // (counted over the whole grouped call: with more matrices than that, the other
+                // launch batches keep the rest of the device busy on their own streams.)
+                int csize = 1;
+                const int room = 2 * sm_count();
+                while (csize < 8 && std::max(merged->count, call_matrices) * csize * 2 <= room) csize *= 2;
+                const size_t dyn = (size_t)2 * r * sizeof(float);
+                if (csize == 1) {
+                    chol_inv_tc_kernel<false><<<merged->count, CT_THREADS, dyn, st>>>(*merged, ca, 1);
+                } else {
+                    cudaLaunchConfig_t cfg{};
+                    cfg.gridDim = dim3((unsigned)(merged->count * csize), 1, 1);
+                    cfg.blockDim = dim3(CT_THREADS, 1, 1);
+                    cfg.dynamicSmemBytes = dyn;
+                    cfg.stream = st;
+                    cudaLaunchAttribute attr[1];
+                    attr[0].id = cudaLaunchAttributeClusterDimension;
+                    attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                    cfg.attrs = attr; cfg.numAttrs = 1;
+                    if (cudaLaunchKernelEx(&cfg, chol_inv_tc_kernel<true>, *merged, ca, csize) != cudaSuccess)
+                        engine_error() = 4;
+                }
+            } else {
+                chol_inv_kernel<<<merged->count, CH_THREADS, CH_SMEM_BYTES, st>>>(*merged, ca);
+            }
             merged->count = 0;
         };
         for (size_t j = i; j < which_cls.size(); ++j) {
@@ -278,7 +311,7 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
 // which = 0: P = orth(Y) (Alg. 1, left-factor step), which = 1: Q = orth(R) (Alg. 1, normalisation step).
 // Tensor engine: the input is an image (w0 holds Y, image r holds R); SIMT engine: fp32 slots.
 void qr_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int which, Batch* merged,
-              cudaStream_t st) {
+              int call_matrices, cudaStream_t st) {
     const int shift_bit = which ? ST_SHIFT_R : ST_SHIFT_L;
     for (int pass = 1; pass <= 3; ++pass) {
         const int only_shift = pass == 3;
@@ -299,7 +332,7 @@ void qr_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int
                 launch_simt(*c.b, r, r, rows, RdPlain{src, 1, r}, RdPlain{src, 1, r}, eg, prof::S_GRAM, st);
             }
         }
-        chol_stage(cls, which_cls, which, pass, merged, st);
+        chol_stage(cls, which_cls, which, pass, merged, call_matrices, st);
         for (int ci : which_cls) {
             ClassRun& c = cls[ci];
             const int r = c.p->r;
@@ -379,7 +412,7 @@ void diag_stage(ClassRun& c, DiagBase db, cudaStream_t st) {
 }
 
 // One step of every class of a group, stage by stage.
-void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, cudaStream_t st) {
+void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, int call_matrices, cudaStream_t st) {
     const Sel sP = sel(W_P), sR = sel(W_R), sQ = sel(W_Q);
     std::vector<int> all, orth;
     for (size_t i = 0; i < cls.size(); ++i) {
@@ -398,7 +431,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, cudaStrea
         else launch_simt(*c.b, p->m, p->r, p->n, RdBuffer{p->n, gb, 0}, RdPlain{sQ, 1, p->r},
                          EpStore{sP, sP, 0, 0, p->r, 0}, prof::S_K1, st);
     }
-    qr_stage(cls, all, 0, merged, st);
+    qr_stage(cls, all, 0, merged, call_matrices, st);
     // Alg. 1, right-factor step:  R = (M + G)^T P
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
@@ -408,14 +441,14 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, cudaStrea
                          EpStore{sR, sR, 0, 0, p->r, 0}, prof::S_K3, st);
     }
     // Alg. 1, normalisation step
-    qr_stage(cls, orth, 1, merged, st);
+    qr_stage(cls, orth, 1, merged, call_matrices, st);
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
         if (p->mode == ORTHDION_MODE_ORTH) continue;
         {
             dim3 grid((unsigned)((p->r + 31) / 32), 1, (unsigned)c.b->count);
             prof::Scope scope(prof::S_COLNORM, st);
-            colnorm_kernel<<<grid, 1024, 0, st>>>(*c.b, p->n, p->r, c.tensor() ? c.sc.ts.cnorm : (int64_t)-1);
+            colnorm_kernel<<<grid, 1024, 0, st>>>(*c.b, p->n, p->r, c.tensor() ? c.sc.ts.cnorm : (int64_t)-1, 0);
         }
         if (c.tensor()) launch_pack(*c.b, sQ, p->n, p->r, c.sc.ts.q, st);
     }
@@ -478,6 +511,7 @@ int orthdion_create(orthdion_t* out, int64_t m, int64_t n, int32_t r, float mu, 
     p->mode = mode;
     p->x_dtype = ORTHDION_DTYPE_BF16; p->g_dtype = ORTHDION_DTYPE_BF16;
     p->engine = tensor_engine_supports(m, n, r) ? ORTHDION_ENGINE_TENSOR : ORTHDION_ENGINE_SIMT;
+    if (p->engine == ORTHDION_ENGINE_SIMT && r > kMaxRankSimt) { delete p; return ORTHDION_ERR_RANK; }
     for (int k = 0; k < 4; ++k) p->passes_set[k] = 0;
     default_passes(p);
     p->diag = 0;
@@ -525,7 +559,11 @@ int orthdion_set_ef(orthdion_t h, float a, float b) {
 
 int orthdion_set_engine(orthdion_t h, int32_t engine) {
     if (!valid(h)) return ORTHDION_ERR_INVALID_ARG;
-    if (engine == ORTHDION_ENGINE_SIMT) { h->engine = engine; return ORTHDION_OK; }
+    if (engine == ORTHDION_ENGINE_SIMT) {
+        if (h->r > kMaxRankSimt) return ORTHDION_ERR_RANK;
+        h->engine = engine;
+        return ORTHDION_OK;
+    }
     if (engine != ORTHDION_ENGINE_TENSOR) return ORTHDION_ERR_INVALID_ARG;
     if (!tensor_engine_supports(h->m, h->n, h->r)) return ORTHDION_ERR_RANK;
     h->engine = engine;
@@ -547,6 +585,7 @@ int orthdion_set_passes(orthdion_t h, int32_t which, int32_t passes) {
 
 int orthdion_set_diagnostics(orthdion_t h, int32_t mask) {
     if (!valid(h) || mask < 0 || mask > 3) return ORTHDION_ERR_INVALID_ARG;
+    if (mask && h->r > kMaxRankSimt) return ORTHDION_ERR_RANK;   // the eigenvalue iteration holds r-vectors in shared memory
     if (mask == 2) mask = 3;      // the buffer norms are reported together with the factor diagnostics
     h->diag = mask;
     return ORTHDION_OK;
@@ -624,14 +663,14 @@ int orthdion_step_grouped(const orthdion_t* hs, int32_t count, void* const* X, f
             for (int l = 0; l < lanes; ++l) cudaStreamWaitEvent(dl->lane[l], dl->fork, 0);
             for (size_t k = 0; k < order.size(); ++k) {
                 std::vector<ClassRun> one(1, cls[order[k]]);
-                run_group(one, merged, db, dl->lane[k % lanes]);
+                run_group(one, merged, db, count, dl->lane[k % lanes]);
             }
             for (int l = 0; l < lanes; ++l) {
                 cudaEventRecord(dl->done[l], dl->lane[l]);
                 cudaStreamWaitEvent(st, dl->done[l], 0);
             }
         } else {
-            run_group(cls, merged, db, st);
+            run_group(cls, merged, db, count, st);
         }
         if (engine_error()) {
             std::fprintf(stderr, "orthdion: tensor map setup failed (%d)\n", engine_error());
@@ -655,6 +694,170 @@ int orthdion_step(orthdion_t h, void* X, float* M, const void* G, float* Q, void
     const void* const gs[1] = {G};
     float* const qs[1] = {Q};
     return orthdion_step_grouped(&h, 1, xs, ms, gs, qs, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+// ---- column-sharded step (Section 2, "FSDP communication") --------------------------------------
+// A matrix split by columns over k ranks, rank j holding X_j, M_j, G_j (m x n_j) and the rows Q_j
+// (n_j x r) of the right factor:  B Q_prev = sum_j B_j Q_j,  R_j = B_j^T P,  R^T R = sum_j R_j^T R_j.
+// The step becomes four local phases with one reduction (a sum over the ranks, made by the
+// caller: NCCL all-reduce on real ranks) of a small buffer between them:
+//   phase 0   Y_j = (M_j + G_j) Q_j                                       -> reduce Y   (m x r)
+//   phase 1   P = orth(Y) (the same on every rank);  R_j = (M_j + G_j)^T P;
+//             ORTH: Gram matrix of R_j;  COLNORM: squared column norms of R_j  -> reduce (r x r | r)
+//   phase 2   ORTH: first CholeskyQR pass of R_j with the reduced Gram matrix, Gram matrix of the
+//             result -> reduce (r x r).   COLNORM: Q_j = R_j / norms, fused update pass: done.
+//   phase 3   ORTH: second pass -> Q_j, fused update pass.
+// The traffic per step is (m + 2 r) r floats (ORTH) or (m + 1) r floats (COLNORM) per rank: the
+// O((m + n) r) of the paper.  The right QR is CholeskyQR2 here; a flagged third pass is not taken.
+namespace {
+struct ShardRun {
+    Batch batch;
+    ClassRun c;
+    Layout lay;
+};
+
+int shard_setup(orthdion_t h, void* X, float* M, const void* G, float* Q, void* workspace, size_t workspace_bytes,
+                ShardRun* sr) {
+    if (!valid(h)) return ORTHDION_ERR_INVALID_ARG;
+    if (h->engine != ORTHDION_ENGINE_TENSOR || h->diag) return ORTHDION_ERR_INVALID_ARG;
+    int e;
+    if ((e = check_ptr(X)) || (e = check_ptr(M)) || (e = check_ptr(G)) || (e = check_ptr(Q))) return e;
+    if (!workspace) return ORTHDION_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return ORTHDION_ERR_WORKSPACE;
+    Batching bt = make_batches(&h, 1);
+    sr->lay = make_layout(&h, 1, bt.scratch_bytes);
+    if (workspace_bytes < sr->lay.total) return ORTHDION_ERR_WORKSPACE;
+    if ((e = ensure_attributes())) return e;
+    char* ws = reinterpret_cast<char*>(workspace);
+    sr->c = ClassRun{h, &sr->batch, scratch_layout(h)};
+    sr->batch.count = 1; sr->batch.pad = 0; sr->batch.scratch_stride = (int64_t)sr->c.sc.bytes;
+    MatWork& w = sr->batch.w[0];
+    w.X = X; w.M = M; w.G = G; w.Q = Q;
+    w.P = reinterpret_cast<float*>(ws + sr->lay.p_off[0]);
+    w.R = reinterpret_cast<float*>(ws + sr->lay.r_off[0]);
+    w.status = reinterpret_cast<int32_t*>(ws + sr->lay.status_off);
+    w.scratch = ws + sr->lay.scratch_off;
+    w.aux0 = 0; w.aux1 = 0;
+    return ORTHDION_OK;
+}
+
+// Gram matrix of the image `src` (rows x r) with its diagonal from the fp32 column squares
+void shard_gram(ShardRun& sr, const ImgRef& src, int64_t rows, cudaStream_t st) {
+    const orthdion_plan* p = sr.c.p;
+    const Sel gram = sel(W_SCRATCH, sr.c.sc.gram);
+    tensor_gram(p->r, p->passes[1], sr.batch, src, rows, gram, 0, st);
+    prof::Scope scope(prof::S_MISC, st);
+    gram_diag_kernel<<<dim3((unsigned)((p->r + 255) / 256), 1, 1), 256, 0, st>>>(
+        sr.batch, gram, p->r, sr.c.sc.ts.colsq, (int)(4 * ((rows + 127) / 128)));
+}
+
+void shard_fused_pass(ShardRun& sr, cudaStream_t st) {
+    const orthdion_plan* p = sr.c.p;
+    const int gb = p->g_dtype == ORTHDION_DTYPE_BF16, xb = p->x_dtype == ORTHDION_DTYPE_BF16;
+    const float cc = 1.f - p->eta * p->wd, dd = p->eta * p->scale;
+    const int fp16 = fused_fp16(p) ? 1 : 0;
+    if (fp16) launch_pack_half(sr.batch, p->n, p->r, sr.c.sc.ts, st);
+    tensor_k5(p->m, p->n, p->r, gb, xb, p->passes[2], p->passes[3], fp16, p->ef_a, p->ef_b, cc, dd, sr.batch,
+              sr.c.sc.ts, st);
+}
+}  // namespace
+
+extern "C" {
+
+int orthdion_shard_phase(orthdion_t h, int32_t phase, void* X, float* M, const void* G, float* Q, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+    ShardRun* sr = new ShardRun();
+    int rc = shard_setup(h, X, M, G, Q, workspace, workspace_bytes, sr);
+    if (rc) { delete sr; return rc; }
+    const orthdion_plan* p = h;
+    const bool orth = p->mode == ORTHDION_MODE_ORTH;
+    if (phase < 0 || phase > (orth ? 3 : 2)) { delete sr; return ORTHDION_ERR_INVALID_ARG; }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
+    const TensorScratch& ts = sr->c.sc.ts;
+    const int r = p->r;
+    std::vector<ClassRun> cls(1, sr->c);
+    const std::vector<int> only(1, 0);
+    Batch* merged = new Batch();
+    engine_error() = 0;
+    if (phase == 0) {
+        {
+            prof::Scope scope(prof::S_MISC, st);
+            init_status_kernel<<<1, 256, 0, st>>>(sr->batch);
+        }
+        tensor_k1(p->m, p->n, r, gb, p->passes[0], sr->batch, ts, st, true);
+    } else if (phase == 1) {
+        // the summed Y sits in the P slot: image and column squares, then the usual left QR
+        launch_pack(sr->batch, sel(W_P), p->m, r, img_view(ts.w0, p->m), st);
+        {
+            prof::Scope scope(prof::S_MISC, st);
+            colsq_blocks_kernel<<<dim3((unsigned)(4 * ((p->m + 127) / 128)), (unsigned)((r + 255) / 256), 1), 256, 0, st>>>(
+                sr->batch, sel(W_P), p->m, r, ts.colsq);
+        }
+        qr_stage(cls, only, 0, merged, 1, st);
+        tensor_k3(p->m, p->n, r, gb, p->passes[0], sr->batch, ts, st);
+        if (orth) {
+            shard_gram(*sr, ts.r, p->n, st);
+        } else {
+            prof::Scope scope(prof::S_COLNORM, st);
+            colnorm_kernel<<<dim3((unsigned)((r + 31) / 32), 1, 1), 1024, 0, st>>>(sr->batch, p->n, r, ts.cnorm, 1);
+        }
+    } else if (phase == 2 && orth) {
+        chol_stage(cls, only, 1, 1, merged, 1, st, true);
+        tc::Dest to_w1 = dest_none(); to_w1.img = img_view(ts.w1, p->n); to_w1.colsq = 1;
+        tc::OutSpec out{};
+        out.ld = r; out.normal = to_w1; out.shifted = to_w1;
+        tensor_apply(r, p->passes[1], sr->batch, ts, ts.r, p->n, out, st);
+        shard_gram(*sr, img_view(ts.w1, p->n), p->n, st);
+    } else if (phase == 2) {
+        {
+            prof::Scope scope(prof::S_COLNORM, st);
+            colnorm_kernel<<<dim3((unsigned)((r + 31) / 32), 1, 1), 1024, 0, st>>>(sr->batch, p->n, r, ts.cnorm, 2);
+        }
+        launch_pack(sr->batch, sel(W_Q), p->n, r, ts.q, st);
+        shard_fused_pass(*sr, st);
+    } else {
+        chol_stage(cls, only, 1, 2, merged, 1, st, true);
+        tc::Dest to_fin = dest_none();
+        to_fin.f32 = sel(W_Q); to_fin.has_f32 = 1; to_fin.img = ts.q;
+        tc::OutSpec out{};
+        out.ld = r; out.normal = to_fin; out.shifted = to_fin;
+        tensor_apply(r, p->passes[1], sr->batch, ts, img_view(ts.w1, p->n), p->n, out, st);
+        shard_fused_pass(*sr, st);
+    }
+    delete merged;
+    delete sr;
+    if (engine_error()) return ORTHDION_ERR_CUDA;
+    cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) {
+        std::fprintf(stderr, "orthdion: launch failed: %s\n", cudaGetErrorString(ce));
+        return ORTHDION_ERR_CUDA;
+    }
+    return ORTHDION_OK;
+}
+
+int orthdion_shard_reduce_buffer(orthdion_t h, int32_t phase, void* workspace, float** buffer, int64_t* count) {
+    if (!valid(h) || !workspace || !buffer || !count) return ORTHDION_ERR_NULL;
+    if (h->engine != ORTHDION_ENGINE_TENSOR) return ORTHDION_ERR_INVALID_ARG;
+    const bool orth = h->mode == ORTHDION_MODE_ORTH;
+    if (phase < 0 || phase > (orth ? 2 : 1)) return ORTHDION_ERR_INVALID_ARG;
+    Batching bt = make_batches(&h, 1);
+    Layout lay = make_layout(&h, 1, bt.scratch_bytes);
+    Scratch sc = scratch_layout(h);
+    char* ws = reinterpret_cast<char*>(workspace);
+    if (phase == 0) {
+        *buffer = reinterpret_cast<float*>(ws + lay.p_off[0]);
+        *count = h->m * (int64_t)h->r;
+    } else if (orth) {
+        *buffer = reinterpret_cast<float*>(ws + lay.scratch_off + sc.gram);
+        *count = (int64_t)h->r * h->r;
+    } else {
+        *buffer = reinterpret_cast<float*>(ws + lay.scratch_off + sc.ts.cnorm);
+        *count = h->r;
+    }
+    return ORTHDION_OK;
 }
 
 }  // extern "C"

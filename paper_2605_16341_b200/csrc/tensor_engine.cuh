@@ -1626,14 +1626,18 @@ inline tc::Dest dest_none() {
 }
 
 // Y = (M + G) Q_prev  -> image w0 (+ column squares)              (Alg. 1, buffer and left-factor steps)
+// partial: the columns at hand are one shard of the matrix; the product goes to the fp32 P slot
+// only, to be summed over the shards before it is orthonormalised.
 inline void tensor_k1(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
-                      cudaStream_t st) {
+                      cudaStream_t st, bool partial = false) {
     launch_pack(b, Sel{W_Q, 0, 0}, n, r, ts.qprev, st);
     tc::GemmArgs g{};
     g.Mrows = (int32_t)m; g.Ncols = r; g.Kdim = (int32_t)n; g.BN = std::min(r, 512);
     g.passes = passes; g.passes2 = 1; g.ld = n; g.n1 = ts.qprev; g.a = no_img(); g.n2 = no_img();
     g.colsq_off = ts.colsq;
-    g.out.normal = dest_none(); g.out.normal.img = img_view(ts.w0, m); g.out.normal.colsq = 1;
+    g.out.normal = dest_none();
+    if (partial) { g.out.normal.f32 = Sel{W_P, 0, 0}; g.out.normal.has_f32 = 1; }
+    else { g.out.normal.img = img_view(ts.w0, m); g.out.normal.colsq = 1; }
     g.out.shifted = g.out.normal; g.out.ld = r;
     if (g_bf16) launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 1>(b, g, prof::S_K1, st);
     else launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K1, st);

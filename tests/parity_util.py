@@ -43,18 +43,28 @@ def rel_max(a, b):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-300))
 
 
-def bf16_steps_apart(x_dev, x_ref32, x_before, slack):
-    """Distance between stored bf16 weights and reference values that are already rounded to bf16,
-    in units of the bf16 spacing at the magnitude of the weight (the larger of the old and the new
-    value, so that a weight that the update happens to cancel is not measured in the tiny steps
-    near zero), after taking off `slack`, the per-entry bound on the error of the single-pass
-    product that feeds the update.  Returns (largest distance, fraction of entries that differ)."""
+def bf16_steps_apart(x_dev, x_ref32, x_before, x_ref_before, slack):
+    """Stored bf16 weights after a step against reference values that are already rounded to bf16.
+
+    bf16 accumulation of updates that are smaller than the spacing is chaotic: an entry whose
+    exact new value sits on a rounding boundary may go either way (about one entry in a thousand
+    per step), and from then on the two copies can sit in different binades, where the same later
+    updates round away in one and are applied in the other.  So the two trajectories are compared
+    where that has not happened yet: on the entries whose value BEFORE the step was identical on
+    both sides, the values after the step may differ by one bf16 step (measured at the larger of the
+    old and the new magnitude) beyond `slack`, the per-entry bound on the error of the single-pass
+    product that feeds the update.  Returns (largest such distance in bf16 steps, fraction of all
+    entries that differ after the step)."""
     a = x_dev.detach().float().cpu().numpy().astype(np.float64)
     b = np.asarray(x_ref32, dtype=np.float64)
-    mag = np.maximum(np.abs(b), np.abs(x_before.detach().float().cpu().numpy().astype(np.float64)))
-    unit = np.maximum(mag, 2.0 ** -126) * 2.0 ** -8        # spacing is between 2^-8 and 2^-7 of the value
+    a0 = x_before.detach().float().cpu().numpy().astype(np.float64)
+    b0 = np.asarray(x_ref_before, dtype=np.float64)
+    mag = np.maximum(np.maximum(np.abs(a), np.abs(b)), np.abs(a0))
+    _, e = np.frexp(np.maximum(mag, 2.0 ** -120))          # mag = f * 2^e, 0.5 <= f < 1
+    step = np.ldexp(1.0, e - 8)                            # bf16 keeps 8 significant bits
     d = np.abs(a - b)
-    return float((np.maximum(d - slack, 0.0) / unit).max()), float(np.count_nonzero(d) / d.size)
+    dist = np.where(a0 == b0, np.maximum(d - slack, 0.0) / step, 0.0)
+    return float(dist.max()), float(np.count_nonzero(d) / d.size)
 
 
 def single_pass_slack(P, Q, eta, scale=1.0, bits=8):

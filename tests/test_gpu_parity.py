@@ -298,7 +298,9 @@ def chain_compare(w, specs, ids, steps, mode, passes=None, seed=0):
         Xb = [x.clone() for x in Xs]
         od.orthdion_step_grouped(od.PointerTable(hs, Xs, Ms, Gd, Qs), ws)
         torch.cuda.synchronize()
-        assert od.orthdion_last_status(hs, ws) == [0] * len(hs)
+        # (a QR may take its third pass: the spike makes B Q_prev less well conditioned as the
+        # warm start aligns with it; that is a flag, not a failure)
+        assert all(f & ~(od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT) == 0 for f in od.orthdion_last_status(hs, ws))
         tol = TOL_STEP if t == 0 else TOL_CHAIN
         for k, i in enumerate(ids):
             spec = specs[i]
@@ -314,12 +316,11 @@ def chain_compare(w, specs, ids, steps, mode, passes=None, seed=0):
             if mode == od.MODE_ORTH:
                 assert np.abs(Qn.T @ Qn - np.eye(spec.r)).max() <= TOL_ORTHO
             assert check_bf16_rounding(Xs[k], Xb[k], P, Qs[k], w.eta, w.wd, 1.0) <= 1.0 + 1e-6
-            # stored weights: the oracle's X', rounded to bf16 like the device's.  An entry whose
-            # exact value lies within the product's error of a rounding boundary may land on the
-            # other side of it, and keeps that one-step distance in later steps.
+            # stored weights: the oracle's X', rounded to bf16 like the device's, on the entries
+            # whose value before the step was the same on both sides
             x_ref = orc.round_to_bf16(ref["X"])
-            ulps, differ = bf16_steps_apart(Xs[k], x_ref, Xb[k], single_pass_slack(P, Qs[k], w.eta))
-            assert ulps <= 2.0 and differ <= 0.02, (spec.name, t, ulps, differ)
+            ulps, differ = bf16_steps_apart(Xs[k], x_ref, Xb[k], Xo, single_pass_slack(P, Qs[k], w.eta))
+            assert ulps <= 1.0 and differ <= 0.02, (spec.name, t, ulps, differ)
             state[k] = [x_ref.astype(np.float64), ref["M"], ref["Q"]]
             worst = dict(dx=max(worst["dx"], e_dx), M=max(worst["M"], e_m), ulps=max(worst["ulps"], ulps),
                          differ=max(worst["differ"], differ))
@@ -367,6 +368,33 @@ def test_single_pass_update_accuracy_on_fp32_weights(mode):
     assert e_factors <= TOL_STEP
     assert e_applied <= 1e-3
     gm.close()
+
+
+# ------------------------------------------------------------------ ranks above 1024
+# The paper's wide-model study runs 16384-wide blocks at rank fraction 0.25 (r = 4096).  These
+# reduced cases take the same path: several 512-column sweeps of the two products with the
+# buffer, Gram matrices of more than four tile rows, and an r x r factor kernel whose lists of
+# tile products exceed one table (r > 1152) and whose row sums span two column blocks.
+@pytest.mark.parametrize("shape,mode", [((2048, 1792, 1536), od.MODE_ORTH), ((1408, 1536, 1280), od.MODE_ORTH),
+                                        ((1408, 1536, 1280), od.MODE_COLNORM)])
+def test_one_step_rank_above_1024(shape, mode):
+    m, n, r = shape
+    spec, X, M, G, Q = make_problem(m, n, r, BF16, BF16, seed=m + n + r)
+    one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_TENSOR)
+
+
+def test_rank_limits():
+    # 4096 is the largest rank; beyond 1024 only the tensor engine (r % 16 == 0) and no diagnostics
+    h = od.orthdion_create(8192, 4096, 4096, 0.95, 0.01, 0.0, od.MODE_ORTH)
+    assert od.orthdion_workspace_bytes(h) > 0
+    with pytest.raises(od.OrthDionError):
+        od.orthdion_set_engine(h, od.ENGINE_SIMT)
+    with pytest.raises(od.OrthDionError):
+        od.orthdion_set_diagnostics(h, 1)
+    od.orthdion_destroy(h)
+    for bad in ((8192, 8192, 4112), (4096, 4096, 1030)):
+        with pytest.raises(od.OrthDionError):
+            od.orthdion_create(*bad, 0.95, 0.01, 0.0, od.MODE_ORTH)
 
 
 def test_tensor_engine_rejects_unsupported_rank():
