@@ -60,6 +60,7 @@ bool same_class(const orthdion_plan* a, const orthdion_plan* b) {
 // depend on r only, so one Cholesky launch can serve matrices of different shapes.
 struct Scratch {
     int64_t gram, linv, tmpA, tmpB;
+    int64_t gram_part;     // partial Gram matrices of a depth-split Gram product (tensor engine, small ranks)
     TensorScratch ts;
     size_t bytes;
 };
@@ -77,6 +78,10 @@ Scratch scratch_layout(const orthdion_plan* p) {
     s.linv = off; off += rr;
     if (p->engine == ORTHDION_ENGINE_TENSOR) {
         off = tensor_scratch_layout(p->m, p->n, p->r, fused_fp16(p), off, &s.ts);
+        // (after everything whose offset must depend on r only)
+        const int parts = std::max(gram_ksplit(p->r, p->m), gram_ksplit(p->r, p->n));
+        s.gram_part = (int64_t)off;
+        if (parts > 1) off += (size_t)parts * rr;
     } else {
         const size_t kr = align_up((size_t)std::max(p->m, p->n) * p->r * 4, 256);
         s.tmpA = off; off += kr;
@@ -324,7 +329,8 @@ void qr_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, int
                 const TensorScratch& ts = c.sc.ts;
                 const ImgRef in = which ? ts.r : img_view(ts.w0, rows);
                 const ImgRef src = pass == 1 ? in : (pass == 2 ? img_view(ts.w1, rows) : img_view(ts.w0, rows));
-                tensor_gram(r, c.p->passes[1], *c.b, src, rows, gram, only_shift ? shift_bit : 0, st);
+                tensor_gram(r, c.p->passes[1], *c.b, src, rows, gram, sel(W_SCRATCH, c.sc.gram_part),
+                            only_shift ? shift_bit : 0, st);
             } else {
                 const Sel in = which ? sel(W_R) : sel(W_P);
                 const Sel src = pass == 1 ? in : (pass == 2 ? sel(W_SCRATCH, c.sc.tmpA) : sel(W_SCRATCH, c.sc.tmpB));
@@ -381,7 +387,7 @@ void diag_stage(ClassRun& c, DiagBase db, cudaStream_t st) {
         diag_init_kernel<<<(b.count * DIAG_STRIDE + 255) / 256, 256, 0, st>>>(b, db);
     }
     if (c.tensor()) {
-        tensor_gram(r, p->passes[1], b, c.sc.ts.q, p->n, gram, 0, st);
+        tensor_gram(r, p->passes[1], b, c.sc.ts.q, p->n, gram, sel(W_SCRATCH, c.sc.gram_part), 0, st);
     } else {
         const Sel sQ = sel(W_Q);
         launch_simt(b, r, r, p->n, RdPlain{sQ, 1, r}, RdPlain{sQ, 1, r}, EpStore{gram, gram, 0, 1, r, 0},
@@ -747,7 +753,7 @@ int shard_setup(orthdion_t h, void* X, float* M, const void* G, float* Q, void* 
 void shard_gram(ShardRun& sr, const ImgRef& src, int64_t rows, cudaStream_t st) {
     const orthdion_plan* p = sr.c.p;
     const Sel gram = sel(W_SCRATCH, sr.c.sc.gram);
-    tensor_gram(p->r, p->passes[1], sr.batch, src, rows, gram, 0, st);
+    tensor_gram(p->r, p->passes[1], sr.batch, src, rows, gram, sel(W_SCRATCH, sr.c.sc.gram_part), 0, st);
     prof::Scope scope(prof::S_MISC, st);
     gram_diag_kernel<<<dim3((unsigned)((p->r + 255) / 256), 1, 1), 256, 0, st>>>(
         sr.batch, gram, p->r, sr.c.sc.ts.colsq, (int)(4 * ((rows + 127) / 128)));

@@ -81,6 +81,9 @@ struct GemmArgs {
     int32_t a_slots, a_slot_bytes;           // A ring
     int32_t epi_bufs;                        // fused pass: 8 KB epilogue buffers per warp (1 or 2)
     int32_t pair;                            // launched as CTA pairs (clusters of two, M = 256 instructions)
+    int32_t ksplit, kb_per_chunk;            // depth split: a tile is computed as `ksplit` partial products over
+                                             // kb_per_chunk depth blocks each, stored split_stride floats apart
+    int64_t split_stride;
     int64_t rscale_off;                      // fp16 fused pass: scratch offset of 1 / (scale of R's plane)
     int64_t ld;                              // leading dimension of M, G, X
     ImgRef a, n1, n2;
@@ -391,7 +394,7 @@ pack_half_kernel(const __grid_constant__ Batch batch, PackHalfArgs a) {
 // ------------------------------------------------------------------------------------------
 // Tile bookkeeping shared by all roles of the GEMM kernel
 // ------------------------------------------------------------------------------------------
-struct TileCoord { int b, mt, nt, n0, bn, kb_end; bool active; };
+struct TileCoord { int b, mt, nt, n0, bn, kb_begin, kb_end, chunk; bool active; };
 // Each role remembers the status word of the matrix it is working on (nothing changes it while
 // the kernel runs), so that only the first tile of a matrix pays for the global load.
 struct StatusCache { int b = -1; int st = 0; };
@@ -403,21 +406,26 @@ template <int EPI>
 __device__ __forceinline__ TileCoord decode_tile(const Batch& batch, const GemmArgs& g, int t, StatusCache& sc,
                                                  int rank) {
     TileCoord c;
-    const int per = g.m_tiles * g.n_tiles;
+    const int per = g.m_tiles * g.n_tiles * g.ksplit;
     c.b = t / per;
-    const int rem = t - c.b * per;
+    int rem = t - c.b * per;
+    c.chunk = 0;
+    if (g.ksplit > 1) { const int tl = rem / g.ksplit; c.chunk = rem - tl * g.ksplit; rem = tl; }
     const int mts = rem / g.n_tiles;
     c.nt = rem - mts * g.n_tiles;
     c.mt = g.pair ? 2 * mts + rank : mts;
     c.n0 = c.nt * g.BN;
     c.bn = min(g.BN, g.Ncols - c.n0);
+    c.kb_begin = 0;
     c.kb_end = g.k_blocks;
     if (g.tri) c.kb_end = min(g.k_blocks, (c.n0 + c.bn + BK - 1) / BK);
+    if (g.ksplit > 1) { c.kb_begin = c.chunk * g.kb_per_chunk; c.kb_end = min(g.k_blocks, c.kb_begin + g.kb_per_chunk); }
     if (c.b != sc.b) { sc.b = c.b; sc.st = *batch.w[c.b].status; }
     const int st = sc.st;
     c.active = !(st & ST_FAILED);
     if (EPI != EPI_K5 && g.out.only_if_shifted && !(st & g.out.shift_bit)) c.active = false;
     if (g.lower_only && c.n0 > (g.pair ? 2 * mts + 1 : c.mt) * BM + BM - 1) c.active = false;
+    if (c.kb_begin >= c.kb_end) c.active = false;
     return c;
 }
 
@@ -537,23 +545,23 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
         if (lane == 0) {
             int as = 0, ns = 0; uint32_t aph = 0, nph = 0;
             // cursor over (tile, depth block) for the A ring
-            int at = tile0, akb = 0; TileCoord ac{}; bool a_done = A_BUF;
+            int at = tile0, akb = -1; TileCoord ac{}; bool a_done = A_BUF;      // akb < 0: tile not decoded yet
             // cursor over (tile, depth block, piece) for the N ring
-            int nt_ = tile0, nkb = 0, npc = 0; TileCoord nc{}; bool n_done = false;
+            int nt_ = tile0, nkb = -1, npc = 0; TileCoord nc{}; bool n_done = false;
             auto a_seek = [&]() {           // make (at, akb) valid or finish
                 while (!a_done) {
                     if (at >= g.total_tiles) { a_done = true; break; }
-                    if (akb == 0) ac = decode_tile<EPI>(batch, g, at, scache, crank);
+                    if (akb < 0) { ac = decode_tile<EPI>(batch, g, at, scache, crank); akb = ac.kb_begin; }
                     if (ac.active && akb < ac.kb_end) break;
-                    at += tstride; akb = 0;
+                    at += tstride; akb = -1;
                 }
             };
             auto n_pieces = [&](int kb) { return NMODE == N_IMG_MN ? mn_pieces(g, kb) : (nc.bn + 127) / 128; };
             auto n_seek = [&]() {           // make (nt_, nkb, npc) valid or finish
                 while (!n_done) {
                     if (nt_ >= g.total_tiles) { n_done = true; break; }
-                    if (nkb == 0 && npc == 0) nc = decode_tile<EPI>(batch, g, nt_, scache, crank);
-                    if (!nc.active || nkb >= nc.kb_end) { nt_ += tstride; nkb = 0; npc = 0; continue; }
+                    if (nkb < 0) { nc = decode_tile<EPI>(batch, g, nt_, scache, crank); nkb = nc.kb_begin; npc = 0; }
+                    if (!nc.active || nkb >= nc.kb_end) { nt_ += tstride; nkb = -1; npc = 0; continue; }
                     if (npc >= n_pieces(nkb)) { ++nkb; npc = 0; continue; }
                     if (NMODE == N_IMG_K && !k_piece_active(g, nc, nkb, npc)) { ++npc; continue; }
                     break;
@@ -579,7 +587,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                     }
                     if (++as == g.a_slots) { as = 0; aph ^= 1; }
                     ++akb;
-                    if (akb >= ac.kb_end) { at += tstride; akb = 0; }
+                    if (akb >= ac.kb_end) { at += tstride; akb = -1; }
                     a_seek();
                     progress = true;
                 }
@@ -654,7 +662,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             // a proxy fence, and a fence per piece stalled the issuer for hundreds of cycles.)
             tc_fence_after();
             const uint32_t dacc = tmem_base + acc * acc_stride;
-            for (int kb = 0; kb < c.kb_end && ok; ++kb) {
+            for (int kb = c.kb_begin; kb < c.kb_end && ok; ++kb) {
                 if (!mbar_wait(a_full0 + 8 * as, aph, abort_flag)) { ok = false; break; }
                 const uint64_t a_kb = a_hi + (a_ring16 + as * a_slot16);
                 if (NMODE == N_IMG_MN) {
@@ -669,7 +677,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                             for (int j = 0; j < nsl; ++j) {
                                 const uint64_t a0 = a_kb + (uint32_t)(sub * per_piece + j) * a_slice16;
                                 const uint64_t a1 = a0 + a_term16;
-                                const uint32_t accum = (kb > 0 || sub > 0 || j > 0) ? 1u : 0u;
+                                const uint32_t accum = (kb > c.kb_begin || sub > 0 || j > 0) ? 1u : 0u;
                                 uint64_t b0 = n_pc + (uint32_t)j * n_slice16;
                                 for (int cc = 0; cc < c.bn; cc += 256) {
                                     const uint32_t idesc = instr_desc((uint32_t)min(256, c.bn - cc), A_MN ? 1u : 0u, 1u, fmt, MROWS);
@@ -711,7 +719,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                 uint64_t a0 = a_hi + (a_ring16 + as * a_slot16);
                                 uint64_t b0 = n_hi + (n_ring16 + ns * n_slot16);
                                 const uint32_t d1 = dacc + ch * 128;
-                                umma_any<PAIR>(d1, a0, b0, idesc2, kb > 0 ? 1u : 0u);
+                                umma_any<PAIR>(d1, a0, b0, idesc2, kb > c.kb_begin ? 1u : 0u);
                                 for (int j = 1; j < nsl; ++j) {
                                     a0 += a_slice16; b0 += n_slice16;
                                     umma_any<PAIR>(d1, a0, b0, idesc2, 1u);
@@ -726,7 +734,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                                                          : smem_desc(sa + A_TERM_BYTES + j * 32, 16, 1024);
                                 const uint64_t b0 = smem_desc(sn + j * 32, 16, 1024);
                                 const uint64_t b1 = smem_desc(sn + A_TERM_BYTES + j * 32, 16, 1024);
-                                const uint32_t accum = (kb > 0 || j > 0) ? 1u : 0u;
+                                const uint32_t accum = (kb > c.kb_begin || j > 0) ? 1u : 0u;
                                 const uint32_t d1 = dacc + ch * 128;
                                 umma_any<PAIR>(d1, a0, b0, idesc, accum);
                                 if (g.passes == 3) {
@@ -776,7 +784,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 const int stw = scache.st;
                 const Dest& d = (g.out.shift_bit && (stw & g.out.shift_bit)) ? g.out.shifted : g.out.normal;
                 const uint32_t taddr = tmem_base + acc * acc_stride + ((uint32_t)(quarter * 32) << 16);
-                float* C = d.has_f32 ? pick(w, d.f32) : nullptr;
+                float* C = d.has_f32 ? pick(w, d.f32) + (int64_t)c.chunk * g.split_stride : nullptr;
                 unsigned char* scr = reinterpret_cast<unsigned char*>(w.scratch);
                 const bool to_img = d.img.off >= 0;
                 float* csq = d.colsq ? reinterpret_cast<float*>(w.scratch + g.colsq_off) +
@@ -1554,7 +1562,9 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     if (pair) g.m_tiles = (g.m_tiles + 1) / 2;      // scheduled row tiles of 256 rows
     g.n_tiles = (g.Ncols + g.BN - 1) / g.BN;
     g.k_blocks = (g.Kdim + tc::BK - 1) / tc::BK;
-    g.total_tiles = b.count * g.m_tiles * g.n_tiles;
+    if (g.ksplit < 1) g.ksplit = 1;
+    if (g.ksplit > 1) g.kb_per_chunk = (g.k_blocks + g.ksplit - 1) / g.ksplit;
+    g.total_tiles = b.count * g.m_tiles * g.n_tiles * g.ksplit;
     const int n1_terms = g.passes == 3 ? 2 : 1, n2_terms = g.passes2 == 3 ? 2 : 1;
     const int bn64 = (g.BN + 63) / 64 * 64;
     const int a_terms = (tc::a_is_buf(AMODE) || g.passes == 3 || (EPI == tc::EPI_K5 && g.passes2 == 3)) ? 2 : 1;
@@ -1657,16 +1667,56 @@ inline void tensor_k3(int64_t m, int64_t n, int r, int g_bf16, int passes, const
     else launch_gemm<tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K3, st);
 }
 
-// Gram = src^T src (src: image of a rows x r matrix); only tiles that touch the lower triangle
-inline void tensor_gram(int r, int passes, const Batch& b, ImgRef src, int64_t rows, Sel gram, int only_shift_bit,
-                        cudaStream_t st) {
+// Depth split of the Gram product.  At small ranks the whole Gram matrix is one output tile whose
+// main loop runs over all rows of the tall matrix on a single CTA (pair): the depth is cut into
+// chunks that run side by side and leave partial sums, which a small kernel adds up in a fixed
+// order.  The number of chunks depends on the rank and the row count only, never on how many
+// matrices a launch holds, so a matrix gets the same bits alone and in any group.
+inline int gram_ksplit(int r, int64_t rows) {
+    if (r > 256) return 1;
+    const int kb = (int)((rows + tc::BK - 1) / tc::BK);
+    const int want = std::min(16, kb / 8);
+    if (want < 2) return 1;
+    const int per = (kb + want - 1) / want;
+    return (kb + per - 1) / per;             // every chunk non-empty
+}
+
+// gram <- sum of the `ksplit` partial matrices at `part` (r x r floats each, r*r apart)
+__global__ void __launch_bounds__(256)
+gram_reduce_kernel(const __grid_constant__ Batch batch, Sel gram, Sel part, int r, int ksplit, int only_shift_bit) {
+    const MatWork& w = batch.w[blockIdx.z];
+    const int st = *w.status;
+    if ((st & ST_FAILED) || (only_shift_bit && !(st & only_shift_bit))) return;
+    const int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x;      // float4 index
+    const int64_t total4 = (int64_t)r * r / 4;
+    if (q >= total4) return;
+    const float4* P = reinterpret_cast<const float4*>(pick(w, part));
+    float4 acc = P[q];
+    for (int s2 = 1; s2 < ksplit; ++s2) {
+        const float4 v = P[(int64_t)s2 * total4 + q];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    reinterpret_cast<float4*>(pick(w, gram))[q] = acc;
+}
+
+// Gram = src^T src (src: image of a rows x r matrix); only tiles that touch the lower triangle.
+// part: scratch for gram_ksplit(r, rows) partial matrices (used when that is more than one).
+inline void tensor_gram(int r, int passes, const Batch& b, ImgRef src, int64_t rows, Sel gram, Sel part,
+                        int only_shift_bit, cudaStream_t st) {
+    const int ksplit = gram_ksplit(r, rows);
     tc::GemmArgs g{};
     g.Mrows = r; g.Ncols = r; g.Kdim = (int32_t)rows; g.BN = std::min(r, 256);
     g.passes = passes; g.passes2 = 1; g.a = src; g.n1 = src; g.n2 = no_img(); g.lower_only = 1;
-    g.out.normal = dest_none(); g.out.normal.f32 = gram; g.out.normal.has_f32 = 1;
+    g.out.normal = dest_none(); g.out.normal.f32 = ksplit > 1 ? part : gram; g.out.normal.has_f32 = 1;
     g.out.shifted = g.out.normal; g.out.ld = r;
     g.out.shift_bit = only_shift_bit; g.out.only_if_shifted = only_shift_bit ? 1 : 0;
+    g.ksplit = ksplit; g.split_stride = (int64_t)r * r;
     launch_gemm<tc::A_IMG_MN, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_GRAM, st);
+    if (ksplit > 1) {
+        prof::Scope scope(prof::S_GRAM, st);
+        dim3 grid((unsigned)(((int64_t)r * r / 4 + 255) / 256), 1, (unsigned)b.count);
+        gram_reduce_kernel<<<grid, 256, 0, st>>>(b, gram, part, r, ksplit, only_shift_bit);
+    }
 }
 
 // dst = src * L^{-T}  (src: image of a rows x r matrix; image linv holds (L^{-1})^T, read MN-major)
