@@ -285,8 +285,13 @@ def run_ours(args):
     tables = [od.PointerTable(hs, Xs, Ms, Gsets[k], Qs) for k in range(args.grad_sets)]
     stream = torch.cuda.current_stream()
 
+    graphs = None
+
     def step(k):
-        od.orthdion_step_grouped(tables[k % args.grad_sets], ws, stream)
+        if graphs is not None:
+            graphs[k % args.grad_sets].replay()
+        else:
+            od.orthdion_step_grouped(tables[k % args.grad_sets], ws, stream)
 
     def barrier():
         if dist is not None:
@@ -298,6 +303,23 @@ def run_ours(args):
     launches_per_step = 0
     if args.warmup > 0:
         launches_per_step = od.orthdion_launch_count() // args.warmup
+    if args.graph:
+        # one CUDA graph per gradient set: a step is then a single graph launch (pays on workloads
+        # whose step is bound by kernel launches; the stage profile is taken without graphs)
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(stream)
+        captured = []
+        for k in range(args.grad_sets):
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=side):
+                od.orthdion_step_grouped(tables[k], ws, torch.cuda.current_stream())
+            captured.append(gr)
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        graphs = captured
+        for k in range(2):
+            step(k)
+        torch.cuda.synchronize()
 
     sampler = ClockSampler(dev) if rank == 0 else None
     if sampler:
@@ -314,6 +336,8 @@ def run_ours(args):
     torch.cuda.synchronize(); barrier()
     t_wall1 = time.time()
     launches = od.orthdion_launch_count() - l0
+    if args.graph:
+        launches = launches_per_step * args.steps      # replayed from the captured graphs, not re-enqueued
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     ms_total = sharding.max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
 
@@ -322,6 +346,7 @@ def run_ours(args):
     # overlapping internal streams of the default configuration would not add up to the step.
     profile_on = not args.no_profile
     stage_ms, ms_step_one_stream = {}, None
+    graphs = None
     if profile_on:
         od.orthdion_set_concurrency(1)
         step(args.warmup + args.steps)                       # settle into the one-stream order
@@ -431,7 +456,7 @@ def run_ours(args):
                                f"bf16 X/G, fp32 M, mode {args.mode}",
                    "engine": args.engine, "l2": "inputs (tens of GB per step) far exceed the 126 MB L2",
                    "grad_sets": args.grad_sets, "replicas": world, "diagnostics": args.diagnostics,
-                   "lanes": args.lanes or DEFAULT_LANES,
+                   "lanes": args.lanes or DEFAULT_LANES, "cuda_graph": bool(args.graph),
                    "diagnostics_summary": diag_summary,
                    "matrices_failed": failed, "matrices_shifted_qr": shifted},
         "clocks": clocks,
@@ -569,6 +594,8 @@ def main():
                     help="on-device diagnostics inside the timed step (0 off, 1 factor diagnostics, 3 plus buffer norms)")
     ap.add_argument("--lanes", type=int, default=None,
                     help="internal streams a grouped call spreads its launch batches over (library default if unset)")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the step from a CUDA graph captured after the warm-up (one per gradient set)")
     ap.add_argument("--grad-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--e2e-chunks", type=int, default=8,

@@ -121,7 +121,10 @@ int orthdion_step(orthdion_t h, void* X, float* M, const void* G, float* Q,
 /* One step for `count` matrices; hs[i] is the plan of matrix i.  X, M, G, Q are HOST arrays of
  * `count` device pointers.  Matrices with equal plan parameters are sorted into packs and every
  * stage runs once per pack (the batching of equal shapes that the paper's appendix on its
- * wide-model study mentions).  Results per matrix are identical to orthdion_step. */
+ * wide-model study mentions).  Results per matrix are identical to orthdion_step.
+ * The call may be recorded into a CUDA graph by stream capture on `stream` and replayed (the
+ * pointers and plan settings are baked into the graph): make one call on the device outside the
+ * capture first, which sets kernel attributes and creates the internal streams. */
 int orthdion_step_grouped(const orthdion_t* hs, int32_t count,
                           void* const* X, float* const* M, const void* const* G, float* const* Q,
                           void* workspace, size_t workspace_bytes, void* stream);
