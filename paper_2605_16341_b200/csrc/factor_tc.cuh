@@ -10,11 +10,12 @@
 // The global loads of the next 32-deep chunk (of this tile or of the next one) are issued before
 // the current chunk is multiplied, so the L2 latency hides behind the work.
 //
-// Right-looking Cholesky with 32-wide panels:
+// Left-looking Cholesky with 32-wide block columns:
+//   column update    W[:, k] -= L[:, <k] L[k, <k]^T                    (tile products, depth 32 k: one
+//                    long pipelined run per 64 rows, every entry of the matrix updated once)
 //   diagonal block   in shared memory: columns scaled by one warp, rank-one updates by all
 //                    threads; then one warp inverts it (needed at the end anyway) in place
 //   panel            rows below  <-  rows below * inv(L_kk)^T          (tile products, depth 32)
-//   trailing update  W22 -= L21 L21^T, lower tiles only                (tile products, depth 32)
 // then the inverse of the factor by combining diagonal blocks pairwise (32, 64, 128, ...):
 //   inv [[A, 0], [B, C]] = [[Ai, 0], [-Ci B Ai, Ci]]                   (tile products)
 // The later passes of a CholeskyQR see a Gram matrix I + E with E tiny; when a rigorous bound on
@@ -23,7 +24,7 @@
 // MULTI form: one matrix per thread-block CLUSTER.  When a launch has fewer matrices than the
 // device has room for CTAs, a lone CTA per matrix leaves most of the device idle while it walks
 // its lists of tile products one after the other.  The CTAs of a cluster share one matrix: every
-// list of independent tile products (panel, trailing update, the two steps of the pairwise
+// list of independent tile products (column update, panel, the two steps of the pairwise
 // inverse) and every copy loop is dealt out over the CTAs, the 32 x 32 diagonal blocks are
 // factored by CTA 0 alone, and phases are separated by cluster barriers.  The matrix stays in
 // global memory (L2); loads of data another CTA of the cluster may have written bypass L1
@@ -436,6 +437,21 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a, int csize) {
 
         for (int k0 = 0; k0 < r; k0 += CT_NB) {
             const int nb = min(CT_NB, r - k0);
+            // Left-looking update of block column k0 with everything to its left:
+            //   W[i][k0 + j] -= sum_{c < k0} W[i][c] W[k0 + j][c],  i >= k0 + j
+            // One tile product per 64 rows with the whole depth k0 in one run (its 32-deep chunks
+            // pipelined), so that every entry of the matrix is read, updated and written once.
+            // (A right-looking trailing update after every panel, 230 short products at r = 512
+            // each with its own round trip for the tile it updates, took 12 % longer on one CTA;
+            // shared by a cluster the two forms are within 4 % of each other, and both forms of the
+            // kernel keep the same one so that a matrix gets the same bits in either.)
+            if (k0 > 0) {
+                run_list([&]() {
+                    for (int i0 = k0; i0 < r; i0 += 64)
+                        add_task(W + (size_t)i0 * r + k0, r, 1, W + (size_t)i0 * r, r, W + (size_t)k0 * r, 1, r,
+                                 min(64, r - i0), nb, 0, k0, -1.f, 1.f, i0 == k0, i0, k0);
+                });
+            }
             // Diagonal block: factored in shared memory by all threads (column scaling by one warp,
             // rank-one update by everybody, two barriers per column), then inverted by one warp
             // (thread c solves L x = e_c with x in registers; L(i, p) are broadcast reads).  The
@@ -493,16 +509,6 @@ chol_inv_tc_kernel(const __grid_constant__ Batch batch, CholArgs a, int csize) {
                     for (int i0 = 0; i0 < s; i0 += 64)
                         add_task(W + (size_t)(t0 + i0) * r + k0, r, 1, W + (size_t)(t0 + i0) * r + k0, r,
                                  W + (size_t)k0 * r + k0, 1, r, min(64, s - i0), nb, 0, nb, 1.f, 0.f, false, 0, 0);
-                });
-                // trailing update: W[t0+i][t0+j] -= sum_c W[t0+i][k0+c] W[t0+j][k0+c], j <= i
-                run_list([&]() {
-                    const int nt = (s + 63) / 64;
-                    for (int ti = 0; ti < nt; ++ti)
-                        for (int tj = 0; tj <= ti; ++tj) {
-                            const int ri = t0 + ti * 64, cj = t0 + tj * 64;
-                            add_task(W + (size_t)ri * r + cj, r, 1, W + (size_t)ri * r + k0, r, W + (size_t)cj * r + k0, 1, r,
-                                     min(64, r - ri), min(64, r - cj), 0, nb, -1.f, 1.f, ti == tj, ri, cj);
-                        }
                 });
             }
         }
