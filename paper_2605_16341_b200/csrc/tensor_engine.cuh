@@ -1417,9 +1417,11 @@ inline size_t tensor_scratch_layout(int64_t m, int64_t n, int32_t r, bool half_p
     ts->rscale = take(16);
     ts->colsq = take(4 * ((kmax + 127) / 128) * (int64_t)r * 4);
     const int pl = half_planes ? 3 : 2;
-    ts->qprev = make_img(take(img_bytes(n, r)), n, r);
     ts->w0 = make_img(take(img_bytes(kmax, r)), kmax, r);
     ts->w1 = make_img(take(img_bytes(kmax, r)), kmax, r);
+    // the image of Q_prev is read by the first product of a step only; w1 is first written after
+    // it (first apply of the left QR, same stream): they share their bytes
+    ts->qprev = make_img(ts->w1.off, n, r);
     ts->p = make_img(take(img_bytes(m, r, pl)), m, r, pl);
     ts->r = make_img(take(img_bytes(n, r, pl)), n, r, pl);
     ts->q = make_img(take(img_bytes(n, r, pl)), n, r, pl);
