@@ -27,7 +27,8 @@
  *  - M and Q are float32.  X and G are float32 or bfloat16 (orthdion_set_dtypes).
  *  - All device pointers must be 16-byte aligned.
  *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
- *    synchronising.  The library allocates no device memory: the caller passes a workspace of
+ *    synchronising.  The device that owns `stream` and the matrices must be the current device
+ *    of the calling thread; per-device set-up (kernel attributes, internal streams) is keyed by it.  The library allocates no device memory: the caller passes a workspace of
  *    at least orthdion_workspace_bytes*() bytes, 256-byte aligned, which must stay untouched
  *    until the enqueued work has finished.  P, R, the status words and the
  *    diagnostic records live in it.
