@@ -60,7 +60,7 @@ bool same_class(const orthdion_plan* a, const orthdion_plan* b) {
 // depend on r only, so one Cholesky launch can serve matrices of different shapes.
 struct Scratch {
     int64_t gram, linv, tmpA, tmpB;
-    int64_t gram_part;     // partial Gram matrices of a depth-split Gram product (tensor engine, small ranks)
+    int64_t gram_part;     // partial results of a depth-split product (tensor engine, small ranks)
     TensorScratch ts;
     size_t bytes;
 };
@@ -80,8 +80,12 @@ Scratch scratch_layout(const orthdion_plan* p) {
         off = tensor_scratch_layout(p->m, p->n, p->r, fused_fp16(p), off, &s.ts);
         // (after everything whose offset must depend on r only)
         const int parts = std::max(gram_ksplit(p->r, p->m), gram_ksplit(p->r, p->n));
+        const int s1 = buffer_ksplit(p->r, p->m, p->n), s3 = buffer_ksplit(p->r, p->n, p->m);
+        size_t part_bytes = parts > 1 ? (size_t)parts * rr : 0;
+        if (s1 > 1) part_bytes = std::max(part_bytes, align_up((size_t)s1 * p->m * p->r * 4, 256));
+        if (s3 > 1) part_bytes = std::max(part_bytes, align_up((size_t)s3 * p->n * p->r * 4, 256));
         s.gram_part = (int64_t)off;
-        if (parts > 1) off += (size_t)parts * rr;
+        off += part_bytes;
     } else {
         const size_t kr = align_up((size_t)std::max(p->m, p->n) * p->r * 4, 256);
         s.tmpA = off; off += kr;
@@ -433,7 +437,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, int call_
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
         const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
-        if (c.tensor()) tensor_k1(p->m, p->n, p->r, gb, p->passes[0], *c.b, c.sc.ts, st);
+        if (c.tensor()) tensor_k1(p->m, p->n, p->r, gb, p->passes[0], *c.b, c.sc.ts, sel(W_SCRATCH, c.sc.gram_part), st);
         else launch_simt(*c.b, p->m, p->r, p->n, RdBuffer{p->n, gb, 0}, RdPlain{sQ, 1, p->r},
                          EpStore{sP, sP, 0, 0, p->r, 0}, prof::S_K1, st);
     }
@@ -442,7 +446,7 @@ void run_group(std::vector<ClassRun>& cls, Batch* merged, DiagBase db, int call_
     for (ClassRun& c : cls) {
         const orthdion_plan* p = c.p;
         const int gb = p->g_dtype == ORTHDION_DTYPE_BF16;
-        if (c.tensor()) tensor_k3(p->m, p->n, p->r, gb, p->passes[0], *c.b, c.sc.ts, st);
+        if (c.tensor()) tensor_k3(p->m, p->n, p->r, gb, p->passes[0], *c.b, c.sc.ts, sel(W_SCRATCH, c.sc.gram_part), st);
         else launch_simt(*c.b, p->n, p->r, p->m, RdBuffer{p->n, gb, 1}, RdPlain{sP, 1, p->r},
                          EpStore{sR, sR, 0, 0, p->r, 0}, prof::S_K3, st);
     }
@@ -793,7 +797,7 @@ int orthdion_shard_phase(orthdion_t h, int32_t phase, void* X, float* M, const v
             prof::Scope scope(prof::S_MISC, st);
             init_status_kernel<<<1, 256, 0, st>>>(sr->batch);
         }
-        tensor_k1(p->m, p->n, r, gb, p->passes[0], sr->batch, ts, st, true);
+        tensor_k1(p->m, p->n, r, gb, p->passes[0], sr->batch, ts, sel(W_SCRATCH, sr->c.sc.gram_part), st, true);
     } else if (phase == 1) {
         // the summed Y sits in the P slot: image and column squares, then the usual left QR
         launch_pack(sr->batch, sel(W_P), p->m, r, img_view(ts.w0, p->m), st);
@@ -803,7 +807,7 @@ int orthdion_shard_phase(orthdion_t h, int32_t phase, void* X, float* M, const v
                 sr->batch, sel(W_P), p->m, r, ts.colsq);
         }
         qr_stage(cls, only, 0, merged, 1, st);
-        tensor_k3(p->m, p->n, r, gb, p->passes[0], sr->batch, ts, st);
+        tensor_k3(p->m, p->n, r, gb, p->passes[0], sr->batch, ts, sel(W_SCRATCH, sr->c.sc.gram_part), st);
         if (orth) {
             shard_gram(*sr, ts.r, p->n, st);
         } else {

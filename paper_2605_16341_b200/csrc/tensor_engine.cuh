@@ -1332,9 +1332,9 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
                 return true;
             };
             Raw r0, r1;
-            fetch(r0, 0);
-            if (c.kb_end > 1) fetch(r1, 1);
-            for (int kb = 0; kb < c.kb_end && ok; kb += 2) {
+            fetch(r0, c.kb_begin);
+            if (c.kb_begin + 1 < c.kb_end) fetch(r1, c.kb_begin + 1);
+            for (int kb = c.kb_begin; kb < c.kb_end && ok; kb += 2) {
                 uint4 t0[2], t1[2];
                 split_raw(r0, t0, t1);
                 if (kb + 2 < c.kb_end) fetch(r0, kb + 2);
@@ -1637,36 +1637,83 @@ inline tc::Dest dest_none() {
     return d;
 }
 
+// Depth split of the two products with the buffer.  With one matrix (or a few) in a call and a
+// small rank, the output has too few 256-row tile pairs for the device (16 for a 4096-wide
+// factor) and every one of them runs over the whole depth: the depth is cut into chunks that run
+// as separate tiles and leave fp32 partial results, which are then added in a fixed order, packed
+// into the operand image and given their column squares by small kernels.  Like the split of the
+// Gram product, the chunk count depends on the plan only (rank, rows of the result, depth), so a
+// matrix gets the same bits alone and in any group; ranks above 256 never split.
+inline int buffer_ksplit(int r, int64_t out_rows, int64_t depth) {
+    if (r > 256) return 1;
+    const int tiles = (int)((out_rows + 255) / 256);
+    const int kb = (int)((depth + tc::BK - 1) / tc::BK);
+    if (tiles >= 37 || kb < 32) return 1;
+    const int want = std::min({8, 74 / tiles, kb / 8});
+    if (want < 2) return 1;
+    const int per = (kb + want - 1) / want;
+    return (kb + per - 1) / per;             // every chunk non-empty
+}
+
+__global__ void gram_reduce_kernel(const __grid_constant__ Batch batch, Sel gram, Sel part, int64_t total4, int ksplit,
+                                   int only_shift_bit);
+
+// after a depth-split product: dst (rows x r fp32) <- sum of the partials, then its image and its
+// column squares per 32-row block
+inline void finish_split_product(const Batch& b, Sel dst, Sel part, int64_t rows, int r, int ksplit, ImgRef img,
+                                 int64_t colsq_off, int stage, cudaStream_t st) {
+    {
+        prof::Scope scope(stage, st);
+        const int64_t total4 = rows * r / 4;
+        dim3 grid((unsigned)((total4 + 255) / 256), 1, (unsigned)b.count);
+        gram_reduce_kernel<<<grid, 256, 0, st>>>(b, dst, part, total4, ksplit, 0);
+    }
+    launch_pack(b, dst, rows, r, img, st);
+    {
+        prof::Scope scope(stage, st);
+        dim3 grid((unsigned)(4 * ((rows + 127) / 128)), (unsigned)((r + 255) / 256), (unsigned)b.count);
+        colsq_blocks_kernel<<<grid, 256, 0, st>>>(b, dst, rows, r, colsq_off);
+    }
+}
+
 // Y = (M + G) Q_prev  -> image w0 (+ column squares)              (Alg. 1, buffer and left-factor steps)
 // partial: the columns at hand are one shard of the matrix; the product goes to the fp32 P slot
 // only, to be summed over the shards before it is orthonormalised.
+// part: scratch for the partial results of a depth split (buffer_ksplit(r, m, n) > 1).
 inline void tensor_k1(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
-                      cudaStream_t st, bool partial = false) {
+                      Sel part, cudaStream_t st, bool partial = false) {
     launch_pack(b, Sel{W_Q, 0, 0}, n, r, ts.qprev, st);
+    const int ksplit = partial ? 1 : buffer_ksplit(r, m, n);
     tc::GemmArgs g{};
     g.Mrows = (int32_t)m; g.Ncols = r; g.Kdim = (int32_t)n; g.BN = std::min(r, 512);
     g.passes = passes; g.passes2 = 1; g.ld = n; g.n1 = ts.qprev; g.a = no_img(); g.n2 = no_img();
     g.colsq_off = ts.colsq;
     g.out.normal = dest_none();
-    if (partial) { g.out.normal.f32 = Sel{W_P, 0, 0}; g.out.normal.has_f32 = 1; }
+    if (ksplit > 1) { g.out.normal.f32 = part; g.out.normal.has_f32 = 1; g.ksplit = ksplit; g.split_stride = m * r; }
+    else if (partial) { g.out.normal.f32 = Sel{W_P, 0, 0}; g.out.normal.has_f32 = 1; }
     else { g.out.normal.img = img_view(ts.w0, m); g.out.normal.colsq = 1; }
     g.out.shifted = g.out.normal; g.out.ld = r;
     if (g_bf16) launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 1>(b, g, prof::S_K1, st);
     else launch_gemm<tc::A_BUF_ROW, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K1, st);
+    // (the sum goes through the fp32 P slot, which holds nothing yet at this point of a step)
+    if (ksplit > 1) finish_split_product(b, Sel{W_P, 0, 0}, part, m, r, ksplit, img_view(ts.w0, m), ts.colsq, prof::S_K1, st);
 }
 
 // R = (M + G)^T P  -> fp32 R slot, image r (+ column squares)     (Alg. 1, right-factor step)
 inline void tensor_k3(int64_t m, int64_t n, int r, int g_bf16, int passes, const Batch& b, const TensorScratch& ts,
-                      cudaStream_t st) {
+                      Sel part, cudaStream_t st) {
+    const int ksplit = buffer_ksplit(r, n, m);
     tc::GemmArgs g{};
     g.Mrows = (int32_t)n; g.Ncols = r; g.Kdim = (int32_t)m; g.BN = std::min(r, 512);
     g.passes = passes; g.passes2 = 1; g.ld = n; g.n1 = ts.p; g.a = no_img(); g.n2 = no_img();
     g.colsq_off = ts.colsq;
-    g.out.normal = dest_none(); g.out.normal.f32 = Sel{W_R, 0, 0}; g.out.normal.has_f32 = 1;
-    g.out.normal.img = ts.r; g.out.normal.colsq = 1;
+    g.out.normal = dest_none(); g.out.normal.has_f32 = 1;
+    if (ksplit > 1) { g.out.normal.f32 = part; g.ksplit = ksplit; g.split_stride = n * r; }
+    else { g.out.normal.f32 = Sel{W_R, 0, 0}; g.out.normal.img = ts.r; g.out.normal.colsq = 1; }
     g.out.shifted = g.out.normal; g.out.ld = r;
     if (g_bf16) launch_gemm<tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 1>(b, g, prof::S_K3, st);
     else launch_gemm<tc::A_BUF_COL, tc::N_IMG_MN, tc::EPI_STORE, 0>(b, g, prof::S_K3, st);
+    if (ksplit > 1) finish_split_product(b, Sel{W_R, 0, 0}, part, n, r, ksplit, ts.r, ts.colsq, prof::S_K3, st);
 }
 
 // Depth split of the Gram product.  At small ranks the whole Gram matrix is one output tile whose
@@ -1683,14 +1730,14 @@ inline int gram_ksplit(int r, int64_t rows) {
     return (kb + per - 1) / per;             // every chunk non-empty
 }
 
-// gram <- sum of the `ksplit` partial matrices at `part` (r x r floats each, r*r apart)
+// dst <- sum of the `ksplit` partial results at `part` (4 * total4 floats each, one after the
+// other), added in the order of the chunks
 __global__ void __launch_bounds__(256)
-gram_reduce_kernel(const __grid_constant__ Batch batch, Sel gram, Sel part, int r, int ksplit, int only_shift_bit) {
+gram_reduce_kernel(const __grid_constant__ Batch batch, Sel gram, Sel part, int64_t total4, int ksplit, int only_shift_bit) {
     const MatWork& w = batch.w[blockIdx.z];
     const int st = *w.status;
     if ((st & ST_FAILED) || (only_shift_bit && !(st & only_shift_bit))) return;
     const int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x;      // float4 index
-    const int64_t total4 = (int64_t)r * r / 4;
     if (q >= total4) return;
     const float4* P = reinterpret_cast<const float4*>(pick(w, part));
     float4 acc = P[q];
@@ -1717,7 +1764,7 @@ inline void tensor_gram(int r, int passes, const Batch& b, ImgRef src, int64_t r
     if (ksplit > 1) {
         prof::Scope scope(prof::S_GRAM, st);
         dim3 grid((unsigned)(((int64_t)r * r / 4 + 255) / 256), 1, (unsigned)b.count);
-        gram_reduce_kernel<<<grid, 256, 0, st>>>(b, gram, part, r, ksplit, only_shift_bit);
+        gram_reduce_kernel<<<grid, 256, 0, st>>>(b, gram, part, (int64_t)r * r / 4, ksplit, only_shift_bit);
     }
 }
 
