@@ -168,6 +168,8 @@ Layout make_layout(const orthdion_t* hs, int32_t count, size_t scratch_bytes) {
 
 // Kernel attributes (dynamic shared-memory limits) belong to a device: they are set once per
 // device ordinal, on the first step call made with that device current.
+signed char g_factor_cluster_max[kMaxDevices] = {};   // written under ensure_attributes()'s lock
+
 int ensure_attributes() {
     static std::mutex mu;
     static signed char state[kMaxDevices] = {};   // 0 unknown, 1 ok, -1 failed
@@ -183,6 +185,24 @@ int ensure_attributes() {
         e = cudaFuncSetAttribute(chol_inv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kMaxRank * 4);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(chol_inv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kMaxRank * 4);
+    // clusters of 16 CTAs are beyond the portable size: allowed per kernel, and used only where the
+    // device says that it can place one
+    g_factor_cluster_max[dev] = 8;
+    if (e == cudaSuccess &&
+        cudaFuncSetAttribute(chol_inv_tc_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(16, 1, 1); cfg.blockDim = dim3(CT_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)2 * kMaxRank * 4;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, chol_inv_tc_kernel<true>, &cfg) == cudaSuccess && clusters >= 1)
+            g_factor_cluster_max[dev] = 16;
+        else
+            (void)cudaGetLastError();
+    }
     if (e == cudaSuccess) e = tensor_engine_set_attributes();
     if (e != cudaSuccess) {
         std::fprintf(stderr, "orthdion: kernel attribute setup failed on device %d: %s\n", dev, cudaGetErrorString(e));
@@ -191,6 +211,12 @@ int ensure_attributes() {
     }
     state[dev] = 1;
     return 0;
+}
+
+int factor_cluster_max() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 8;
+    return g_factor_cluster_max[dev] == 16 ? 16 : 8;
 }
 
 // ---- internal streams of the grouped step ---------------------------------------------------
@@ -273,12 +299,14 @@ void chol_stage(std::vector<ClassRun>& cls, const std::vector<int>& which_cls, i
             prof::Scope scope(prof::S_CHOL, st);
             if (lead.tensor()) {
                 // Fewer matrices than the device has room for CTAs (two per multiprocessor): share
-                // each matrix among the CTAs of a cluster (2, 4 or 8).
+                // each matrix among the CTAs of a cluster (2, 4 or 8; 16 from rank 512 up, where the
+                // tile lists are long enough to feed them and the device can place such a cluster).
                 // (counted over the whole grouped call: with more matrices than that, the other
                 // launch batches keep the rest of the device busy on their own streams.)
                 int csize = 1;
                 const int room = 2 * sm_count();
-                while (csize < 8 && std::max(merged->count, call_matrices) * csize * 2 <= room) csize *= 2;
+                const int cmax = r >= 512 ? factor_cluster_max() : 8;
+                while (csize < cmax && std::max(merged->count, call_matrices) * csize * 2 <= room) csize *= 2;
                 const size_t dyn = (size_t)2 * r * sizeof(float);
                 if (csize == 1) {
                     chol_inv_tc_kernel<false><<<merged->count, CT_THREADS, dyn, st>>>(*merged, ca, 1);
