@@ -487,7 +487,7 @@ def run_ours(args):
 # dram__bytes_write.sum of one launch) on a 4-layer case of the same kernel: 6.782 GB over
 # 469.8 M elements.  Traffic grows in proportion to the elements, so a step's traffic is this
 # figure x its elements.  Set to None whenever the kernel changes until the counters are retaken.
-MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.43}
+MEASURED_DRAM_BYTES_PER_ELEMENT = {("cfg4", "k5_feedback_update"): 14.44}
 
 
 def run_e2e(args, od, w, dev, stream, tables, ws, Xs, Gsets, world, dist):
