@@ -45,10 +45,12 @@ enum NMode : int { N_IMG_K = 0, N_IMG_MN = 1 };
 enum EpiMode : int { EPI_STORE = 0, EPI_K5 = 1 };
 
 __host__ __device__ constexpr bool a_is_buf(int amode) { return amode == A_BUF_ROW || amode == A_BUF_COL; }
-// Eight epilogue warps (two per tensor-memory lane quarter, splitting the columns) wherever the
-// epilogue is a large share of a tile's time: the fused pass and the image-to-image products of
-// the QR.  The products that form B have sixteen transform warps already and a short epilogue.
-__host__ __device__ constexpr int epi_warps(int amode, int epi) { return (epi == EPI_K5 || !a_is_buf(amode)) ? 8 : 4; }
+// Eight epilogue warps (two per tensor-memory lane quarter, splitting the columns) for the fused
+// pass, whose epilogue is most of a tile's time.  Everywhere else four: the products that form B
+// have sixteen transform warps already, and the image-to-image products of the QR do better with
+// the 32 KB of staging that four more warps would take spent on a third A slot (they are bound by
+// the latency of their operand tiles: measured apply 10.3 -> 9.4 ms, Gram 8.85 -> 8.5 ms).
+__host__ __device__ constexpr int epi_warps(int amode, int epi) { (void)amode; return epi == EPI_K5 ? 8 : 4; }
 __host__ __device__ constexpr int gemm_threads(int amode, int epi) {
     return 32 * (2 + epi_warps(amode, epi) + (a_is_buf(amode) ? NUM_XF_WARPS : 0));
 }
@@ -967,8 +969,7 @@ gemm_kernel(const __grid_constant__ Batch batch, const __grid_constant__ GemmArg
             // Fused error feedback and weight update.  Warp (quarter, half) owns rows
             // 32*quarter.. of the tile and columns 64*half.., in two slabs of 32 x 32.  The two
             // accumulator slabs go through a swizzled staging block so that global accesses run
-            // along rows (8 lanes x 16 bytes per row).  The producer warp has already asked for the
-            // tile's M, G, X in L2, so the loads of a slab return with L2 latency.
+            // along rows (8 lanes x 16 bytes per row).
             const int half = (warp - 2) / 4;
             auto next_tile = [&](int t) {
                 for (t += tstride; t < g.total_tiles; t += tstride)
@@ -1572,6 +1573,8 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     const int a_terms = (tc::a_is_buf(AMODE) || g.passes == 3 || (EPI == tc::EPI_K5 && g.passes2 == 3)) ? 2 : 1;
     g.a_slot_bytes = a_terms * tc::A_TERM_BYTES;
     g.a_slots = tc::A_RING_BYTES / g.a_slot_bytes;
+    // image-to-image products: a third two-term slot (the N ring then holds three pieces as well)
+    if (EPI == tc::EPI_STORE && !tc::a_is_buf(AMODE)) g.a_slots = std::min(tc::MAX_A_SLOTS, 6 * tc::A_TERM_BYTES / g.a_slot_bytes);
     g.epi_bufs = 1;
     if (EPI == tc::EPI_K5) {
         // the fused pass needs little MMA time per tile: two slots per ring, and (bf16 G and X,
