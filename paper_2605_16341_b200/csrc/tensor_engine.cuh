@@ -1577,10 +1577,9 @@ inline void launch_gemm(const Batch& b, tc::GemmArgs g, int stage, cudaStream_t 
     if (EPI == tc::EPI_STORE && !tc::a_is_buf(AMODE)) g.a_slots = std::min(tc::MAX_A_SLOTS, 6 * tc::A_TERM_BYTES / g.a_slot_bytes);
     g.epi_bufs = 1;
     if (EPI == tc::EPI_K5) {
-        // the fused pass needs little MMA time per tile: two slots per ring, and (bf16 G and X,
-        // single-pass operands) a second epilogue buffer per warp instead
+        // the fused pass: 64 KB of A slots (four single-term ones or two two-term ones) and one
+        // epilogue buffer per warp (a second one, paid for with ring slots, measured slower)
         g.a_slots = (a_terms == 1) ? 4 : 2;
-        if (XG == 3 && a_terms == 1) g.epi_bufs = 1;
     }
     if (NMODE == tc::N_IMG_MN) {
         if (pair) {
