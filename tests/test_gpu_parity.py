@@ -250,6 +250,42 @@ def test_grouped_matches_single_and_is_deterministic(engine):
         od.orthdion_destroy(h)
 
 
+@pytest.mark.parametrize("shape", [(128, 192, 64), (512, 640, 512)])
+@pytest.mark.parametrize("count", [150, 40])
+def test_factor_kernel_forms_agree_bit_for_bit(shape, count):
+    """The r x r factor kernel runs one CTA per matrix when a call holds more matrices than the
+    device has room for clusters, and shares a matrix among the 2, 4, 8 or (from rank 512) 16 CTAs
+    of a cluster when it holds fewer.  Every form does the same arithmetic in the same order: a
+    matrix stepped inside a call of 150 (one CTA each) or 40 (clusters of two) gets the bits it
+    gets when stepped alone (the largest cluster)."""
+    m, n, r = shape
+    specs, st, Gs = [], [], []
+    for i in range(count):
+        spec, X, M, G, Q = make_problem(m, n, r, BF16, BF16, seed=7000 + i)
+        specs.append(spec); st.append((X, M, Q)); Gs.append(G)
+    h = od.orthdion_create(m, n, r, 0.95, 0.01, 0.0, od.MODE_ORTH)
+    od.orthdion_set_dtypes(h, BF16, BF16)
+    hs = [h] * count
+    dev = [tuple(t.cuda() for t in s) for s in st]
+    Gd = [g.cuda() for g in Gs]
+    ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
+    table = od.PointerTable(hs, [d[0] for d in dev], [d[1] for d in dev], Gd, [d[2] for d in dev])
+    od.orthdion_step_grouped(table, ws)
+    torch.cuda.synchronize()
+    flags = od.orthdion_last_status(hs, ws)
+    assert all(f & ~(od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT) == 0 for f in flags)
+    for i in (0, count // 2, count - 1):
+        gm = GpuMatrix(specs[i], *st[i], mu=0.95, eta=0.01, engine=od.ENGINE_TENSOR)
+        gm.step(Gs[i])
+        assert gm.status() == flags[i]
+        assert torch.equal(gm.X, dev[i][0]) and torch.equal(gm.M, dev[i][1]) and torch.equal(gm.Q, dev[i][2])
+        P, R = od.orthdion_get_factors(hs, i, ws, (m, n, r))
+        P1, R1 = gm.factors()
+        assert torch.equal(P, P1) and torch.equal(R, R1)
+        gm.close()
+    od.orthdion_destroy(h)
+
+
 @pytest.mark.parametrize("engine", ENGINES, ids=ENGINE_IDS)
 def test_state_is_only_m_and_q(engine):
     # 4 steps in one go == 2 steps, state copied out and back, 2 more steps (bitwise)
