@@ -54,6 +54,8 @@ def test_host_argument_checks(L):
     assert ws >= 4 * (256 + 512) * 16
     # null pointers are rejected before anything is enqueued
     assert L.orthdion_step(h, None, None, None, None, None, 0, None) == -3
+    assert L.orthdion_set_concurrency(0) == -1 and L.orthdion_set_concurrency(9) == -1
+    assert L.orthdion_set_concurrency(4) == 0   # the default
     assert L.orthdion_destroy(h) == 0
     assert L.orthdion_destroy(h) == -1          # stale handle is recognised
     assert b.orthdion_version().startswith("orthdion")

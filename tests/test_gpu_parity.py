@@ -250,6 +250,44 @@ def test_grouped_matches_single_and_is_deterministic(engine):
         od.orthdion_destroy(h)
 
 
+def test_internal_streams_change_no_bit():
+    """A grouped call runs its launch batches on 1 to 8 internal streams: two steps of five classes
+    (twelve matrices) leave the same bits whatever the number of streams."""
+    shapes = [(256, 384, 32)] * 3 + [(384, 256, 64)] * 2 + [(520, 392, 48)] * 3 + [(128, 1024, 16)] * 2 + \
+             [(640, 384, 256)] * 2
+    probs = [make_problem(m, n, r, BF16, BF16, seed=300 + i) for i, (m, n, r) in enumerate(shapes)]
+    hs = []
+    for spec, *_ in probs:
+        h = od.orthdion_create(spec.m, spec.n, spec.r, 0.95, 0.01, 0.0, od.MODE_ORTH)
+        od.orthdion_set_dtypes(h, BF16, BF16)
+        hs.append(h)
+    outs = []
+    try:
+        for lanes in (1, 2, 4, 8):
+            od.orthdion_set_concurrency(lanes)
+            Xs = [p[1].cuda() for p in probs]; Ms = [p[2].cuda() for p in probs]
+            Gd = [p[3].cuda() for p in probs]; Qs = [p[4].cuda() for p in probs]
+            ws = poisoned_workspace(od.orthdion_workspace_bytes_grouped(hs))
+            table = od.PointerTable(hs, Xs, Ms, Gd, Qs)
+            for _ in range(2):
+                od.orthdion_step_grouped(table, ws)
+            torch.cuda.synchronize()
+            assert od.orthdion_last_status(hs, ws) == [0] * len(hs)
+            outs.append((Xs, Ms, Qs))
+    finally:
+        od.orthdion_set_concurrency(4)
+    for other in outs[1:]:
+        for k in range(3):
+            for a, b in zip(outs[0][k], other[k]):
+                assert torch.equal(a, b)
+    with pytest.raises(Exception):
+        od.orthdion_set_concurrency(0)
+    with pytest.raises(Exception):
+        od.orthdion_set_concurrency(9)
+    for h in hs:
+        od.orthdion_destroy(h)
+
+
 @pytest.mark.parametrize("shape", [(128, 192, 64), (512, 640, 512)])
 @pytest.mark.parametrize("count", [150, 40])
 def test_factor_kernel_forms_agree_bit_for_bit(shape, count):
