@@ -69,3 +69,41 @@ def test_grouped_workspace_is_at_least_the_sum_of_factors(L):
     assert need >= max(b.orthdion_workspace_bytes(h) for h in hs)
     for h in hs:
         b.orthdion_destroy(h)
+
+
+def test_default_pass_counts_follow_dtypes_and_feedback_form(L):
+    """The pass counts of the fused feedback/update product follow the plan until the caller fixes
+    them: one fp16 pass each for bf16 weights in the momentum form (|b| <= 0.1 |a|), three bf16
+    passes for P R^T in the residual form a = b and for fp32 weights.  The fp16 form shows in the
+    workspace: P, R and Q then carry a third operand plane (2 bytes per entry)."""
+    m, n, r = 512, 768, 64
+    planes = 2 * (m + 2 * n) * r                      # bytes of the fp16 planes (rows are multiples of 128)
+
+    def plan():
+        h = ctypes.c_void_p()
+        assert L.orthdion_create(ctypes.byref(h), m, n, r, ctypes.c_float(0.95), ctypes.c_float(0.01),
+                                 ctypes.c_float(0.0), 0) == 0
+        return h
+
+    h = plan()
+    fused = L.orthdion_workspace_bytes(h)             # defaults: bf16 weights, momentum form (a = 1, b = 0.05): 1, 1
+    assert L.orthdion_set_dtypes(h, 0, 0) == 0        # fp32 weights and gradients: 3, 3
+    base = L.orthdion_workspace_bytes(h)
+    assert fused - base == planes
+    assert L.orthdion_set_dtypes(h, 1, 1) == 0
+    assert L.orthdion_workspace_bytes(h) == fused
+    assert L.orthdion_set_ef(h, ctypes.c_float(0.95), ctypes.c_float(0.95)) == 0      # residual form: 3, 1
+    assert L.orthdion_workspace_bytes(h) == base
+    assert L.orthdion_set_ef(h, ctypes.c_float(1.0), ctypes.c_float(0.05)) == 0
+    assert L.orthdion_workspace_bytes(h) == fused
+    assert L.orthdion_set_passes(h, 2, 3) == 0        # fixed by the caller: stays through later changes
+    assert L.orthdion_workspace_bytes(h) == base
+    assert L.orthdion_set_dtypes(h, 1, 1) == 0
+    assert L.orthdion_workspace_bytes(h) == base
+    assert L.orthdion_set_passes(h, 2, 0) == 0        # handed back to the rule
+    assert L.orthdion_workspace_bytes(h) == fused
+    assert L.orthdion_set_dtypes(h, 0, 1) == 0        # fp32 weights again
+    assert L.orthdion_workspace_bytes(h) == base
+    assert L.orthdion_set_passes(h, 2, 1) == 0 and L.orthdion_set_passes(h, 3, 1) == 0
+    assert L.orthdion_workspace_bytes(h) == fused     # asked for explicitly
+    assert L.orthdion_destroy(h) == 0
