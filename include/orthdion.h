@@ -28,10 +28,10 @@
  *  - All device pointers must be 16-byte aligned.
  *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
  *    synchronising.  The device that owns `stream` and the matrices must be the current device
- *    of the calling thread; per-device set-up (kernel attributes, internal streams) is keyed by it.  The library allocates no device memory: the caller passes a workspace of
- *    at least orthdion_workspace_bytes*() bytes, 256-byte aligned, which must stay untouched
- *    until the enqueued work has finished.  P, R, the status words and the
- *    diagnostic records live in it.
+ *    of the calling thread; per-device set-up (kernel attributes, internal streams) is keyed by
+ *    it.  The library allocates no device memory: the caller passes a workspace of at least
+ *    orthdion_workspace_bytes*() bytes, 256-byte aligned, which must stay untouched until the
+ *    enqueued work has finished.  P, R, the status words and the diagnostic records live in it.
  *  - Return value: 0 on success, a negative ORTHDION_ERR_* code when the host rejects the
  *    arguments (nothing is enqueued then).  Numerical conditions never trap: they are reported
  *    per matrix through status flags in the workspace (orthdion_last_status).  A matrix whose
