@@ -288,8 +288,9 @@ def test_internal_streams_change_no_bit():
         od.orthdion_destroy(h)
 
 
-@pytest.mark.parametrize("shape", [(128, 192, 64), (512, 640, 512)])
-@pytest.mark.parametrize("count", [150, 40])
+# (the last case also has more matrices of one plan than a launch batch holds: two batches)
+@pytest.mark.parametrize("shape,count", [((128, 192, 64), 150), ((128, 192, 64), 40), ((512, 640, 512), 150),
+                                         ((512, 640, 512), 40), ((64, 64, 16), 300)])
 def test_factor_kernel_forms_agree_bit_for_bit(shape, count):
     """The r x r factor kernel runs one CTA per matrix when a call holds more matrices than the
     device has room for clusters, and shares a matrix among the 2, 4, 8 or (from rank 512) 16 CTAs
