@@ -458,6 +458,48 @@ def test_one_step_rank_above_1024(shape, mode):
     one_step_compare(spec, X, M, G, Q, mode=mode, engine=od.ENGINE_TENSOR)
 
 
+def test_one_step_at_the_largest_rank():
+    """r = 4096 (the paper's 16384-wide blocks at rank fraction 0.25) on a 6144 x 8192 matrix.  The
+    float64 oracle's QR would take minutes here; the results are held to what defines them, formed
+    in float64 on the device: P and Q orthonormal, R = B^T P, col(P) = col(B Q_prev), Q R-factor
+    upper triangular with positive diagonal, M' = a B - b P R^T."""
+    m, n, r = 6144, 8192, 4096
+    g = torch.Generator(device="cuda").manual_seed(5)
+    X = (0.02 * torch.randn(m, n, generator=g, device="cuda")).to(BF16)
+    M = 0.3 * torch.randn(m, n, generator=g, device="cuda")
+    G = torch.randn(m, n, generator=g, device="cuda").to(BF16)
+    Q0 = torch.linalg.qr(torch.randn(n, r, generator=g, device="cuda", dtype=torch.float64))[0].float().contiguous()
+    h = od.orthdion_create(m, n, r, 0.95, 0.01, 0.0, od.MODE_ORTH)
+    ws = poisoned_workspace(od.orthdion_workspace_bytes(h))
+    Xd, Md, Qd = X.clone(), M.clone(), Q0.clone()
+    od.orthdion_step(h, Xd, Md, G, Qd, ws)
+    torch.cuda.synchronize()
+    st = od.orthdion_last_status([h], ws)[0]
+    assert st & ~(od.STATUS_SHIFTED_LEFT | od.STATUS_SHIFTED_RIGHT) == 0
+    P, R = od.orthdion_get_factors([h], 0, ws, (m, n, r))
+    B = M.double() + G.double()
+    P64, R64, Q64 = P.double(), R.double(), Qd.double()
+    eye = torch.eye(r, device="cuda", dtype=torch.float64)
+    assert (P64.T @ P64 - eye).abs().max().item() <= TOL_ORTHO
+    assert (Q64.T @ Q64 - eye).abs().max().item() <= TOL_ORTHO
+    Rref = B.T @ P64
+    assert ((R64 - Rref).norm() / Rref.norm()).item() <= TOL_STEP
+    Y = B @ Q0.double()
+    assert ((Y - P64 @ (P64.T @ Y)).norm() / Y.norm()).item() <= TOL_STEP          # col(Y) inside col(P)
+    T = Q64.T @ R64                                                                    # R = Q T
+    assert ((R64 - Q64 @ T).norm() / R64.norm()).item() <= TOL_STEP
+    assert (torch.tril(T, -1).norm() / T.norm()).item() <= TOL_STEP and (torch.diagonal(T) > 0).all()
+    Mref = B - 0.05 * (P64 @ R64.T)
+    assert ((Md.double() - Mref).norm() / Mref.norm()).item() <= TOL_STEP
+    dX = -0.01 * (P64 @ Q64.T)
+    got = Xd.double() - X.double()
+    # stored bf16 weights: within one bf16 step of the exact update (plus the single-pass bound)
+    ulp = X.double().abs().clamp_min(2.0 ** -126) * 2.0 ** -7
+    slack = 0.01 * 2.0 ** -8 * (P64.abs() @ Q64.abs().T)
+    assert (((got - dX).abs() - slack) / ulp).max().item() <= 1.0 + 1e-6
+    od.orthdion_destroy(h)
+
+
 def test_rank_limits():
     # 4096 is the largest rank; beyond 1024 only the tensor engine (r % 16 == 0) and no diagnostics
     h = od.orthdion_create(8192, 4096, 4096, 0.95, 0.01, 0.0, od.MODE_ORTH)
